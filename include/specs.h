@@ -1,0 +1,204 @@
+/*
+ * specs.h -- C ABI of the B200 (sm_100a) block-scoring library for SPECS
+ * (arxiv 2506.15733, "Faster Test-Time Scaling through Speculative Drafts and
+ * Dynamic Switching").
+ *
+ * One beam step of the method scores n drafted candidate blocks per problem:
+ * the target model's LM head gives log pi_target of every drafted token, the
+ * per-block sums enter the score of Eq. (1) together with the generator's own
+ * log-probabilities and the process-reward score, Algorithm 2 (SubSample)
+ * samples one candidate with probability proportional to exp(S_i), and Step III
+ * of Algorithm 1 decides whether the draft model may generate the next step.
+ *
+ * General rules for every call below
+ *   - Pointers are DEVICE pointers unless their name starts with h_.  The
+ *     caller owns every buffer; nothing passed in is retained after the work
+ *     enqueued by the call has finished.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls validate their arguments on the host, enqueue work on the stream
+ *     and return without synchronising, unless stated otherwise.
+ *   - The return value is a specs_status.  On any value other than SPECS_OK
+ *     nothing was launched and the outputs are untouched.
+ *   - Conditions found on the device (a drafted id outside [0, V), a bounded
+ *     wait inside a kernel that expired) never trap: they set bits in a device
+ *     status word that specs_device_status() reads.
+ *   - One context serves one stream at a time.
+ */
+#ifndef SPECS_H_
+#define SPECS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct specs_ctx specs_ctx;
+
+typedef enum specs_status {
+    SPECS_OK = 0,
+    SPECS_ERR_NULL = 1,            /* a required pointer is NULL */
+    SPECS_ERR_SHAPE = 2,           /* rows < 0, d <= 0, d % 8 != 0, V <= 0, B < 0, P < 0, ... */
+    SPECS_ERR_ALIGN = 3,           /* hidden / W_vocab / workspace not 16-byte aligned */
+    SPECS_ERR_WORKSPACE = 4,       /* workspace smaller than specs_score_workspace_bytes() */
+    SPECS_ERR_OFFSETS = 5,         /* h_ offsets not starting at 0 / decreasing / not ending at the total */
+    SPECS_ERR_ARCH = 6,            /* device is not compute capability 10.x */
+    SPECS_ERR_CUDA = 7,            /* a CUDA runtime or driver call failed */
+    SPECS_ERR_DEVICE_TIMEOUT = 8,  /* device status: a bounded wait in a kernel expired */
+    SPECS_ERR_TOKEN_RANGE = 9,     /* device status: some drafted id was outside [0, V) */
+    SPECS_ERR_LIMIT = 10           /* a size exceeds a documented maximum */
+} specs_status;
+
+/* Bits of the device status word returned by specs_device_status(). */
+#define SPECS_DEV_TIMEOUT      0x1u
+#define SPECS_DEV_TOKEN_RANGE  0x2u
+
+/* Scoring engines (see specs_set_engine). */
+#define SPECS_ENGINE_TCGEN05 0   /* tensor-core path: TMA + tcgen05.mma + TMEM, fused epilogue (default) */
+#define SPECS_ENGINE_SIMT    1   /* plain CUDA-core kernel; a bring-up and bisecting aid, never chosen automatically */
+
+/* Human-readable name of a status value (static string, never NULL). */
+const char* specs_status_string(int status);
+
+/* Create / destroy a context on CUDA device `device`.  Creation allocates a few
+ * bytes of device memory (the status word) and looks up the driver's tensor-map
+ * encoder; it fails with SPECS_ERR_ARCH on anything but sm_100-class devices. */
+int specs_create(specs_ctx** out, int device);
+int specs_destroy(specs_ctx* ctx);
+
+/* Select the scoring engine for later specs_score_blocks calls on this context. */
+int specs_set_engine(specs_ctx* ctx, int engine);
+
+/* Number of SMs the context schedules over (also the persistent grid size). */
+int specs_sm_count(const specs_ctx* ctx);
+
+/* Bytes of scratch specs_score_blocks needs for these sizes.  It holds one
+ * (running max, sum of exponentials, drafted-token logit) triple per row and per
+ * vocabulary split -- a few hundred KB per 148 row tiles -- and never anything
+ * proportional to rows x V: the logits themselves exist only in tensor memory. */
+size_t specs_score_workspace_bytes(const specs_ctx* ctx, int64_t rows, int32_t d, int32_t V);
+
+/* log pi_target of every drafted token and of every drafted block
+ * (Section 2: "computing logits of each token" of a drafted block with the
+ * target model; Appendix E.3: only the newly drafted tokens are scored; Eq. (1):
+ * the block probability is the product over its tokens).
+ *
+ *   hidden        bf16 [rows, d] row-major: the target's final hidden state (after
+ *                 its last norm) at the position that predicts each drafted token.
+ *   W_vocab       bf16 [V, d] row-major LM-head weight (no bias, temperature 1).
+ *   token_ids     int32 [rows]: the drafted ids.  An id outside [0, V) yields NaN
+ *                 for that token and sets SPECS_DEV_TOKEN_RANGE.
+ *   block_offsets int64 [B+1] on the device: block i owns rows [off[i], off[i+1]);
+ *                 off[0] = 0, non-decreasing, off[B] = rows (caller's contract; an
+ *                 empty block has log-probability 0).
+ *   tok_logprob   float [rows] out.   blk_logprob float [B] out (may be NULL).
+ *   blk_logprob_f64 double [B] out (may be NULL): the same sums before rounding.
+ *   workspace     scratch of at least specs_score_workspace_bytes(), 16-byte aligned.
+ *
+ * Requirements: d % 8 == 0 (rows of both matrices must start on 16-byte
+ * boundaries), hidden and W_vocab 16-byte aligned.  rows == 0 is a valid no-op
+ * (block sums are then written as 0). */
+int specs_score_blocks(specs_ctx* ctx, const void* hidden, const void* W_vocab,
+                       const int32_t* token_ids, const int64_t* block_offsets,
+                       int64_t rows, int32_t d, int32_t V, int32_t B,
+                       float* tok_logprob, float* blk_logprob, double* blk_logprob_f64,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Segmented sum of a per-token array over the blocks (the same reduction as inside
+ * specs_score_blocks; used for the generator's own per-token log-probabilities,
+ * the denominator of Eq. (1)).  Accumulates in double.  out / out_f64 may each be
+ * NULL but not both. */
+int specs_block_sums(specs_ctx* ctx, const float* per_token, const int64_t* block_offsets,
+                     int32_t B, float* out, double* out_f64, void* cuda_stream);
+
+/* SubSample (Algorithm 2) for P problems at once, fused with the switch test.
+ *
+ *   S_i = (blk_lp_target[i] - blk_lp_gen[i]) + beta * reward[i]            (Eq. 1)
+ *   weights[i] = exp(S_i) / sum over the problem's candidates of exp(S_j)  (Algorithm 2)
+ *   chosen[p]  = argmax_i (S_i - log(-log uniforms[i])), index local to the problem,
+ *                lowest index on exact ties: an exact draw from `weights` when the
+ *                uniforms are i.i.d. U(0,1); -1 for a problem without candidates.
+ *   accept[p]  = 1 iff max_i reward[i] > tau (Algorithm 1, Step III), 0 otherwise.
+ *
+ *   blk_lp_gen == NULL means the blocks came from the target itself
+ *   (pi_gen = pi_target): the ratio drops out and S_i = beta * reward[i];
+ *   blk_lp_target may then be NULL too.
+ *   cand_offsets int32 [P+1] on the device: problem p owns blocks
+ *   [cand_offsets[p], cand_offsets[p+1]).
+ *   uniforms float [total candidates], each strictly inside (0,1); values outside
+ *   are clamped to [2^-25, 1 - 2^-24].
+ *   accept may be NULL (then tau is ignored).  weights may be NULL.
+ *   Scores, the maximum, the normaliser and the perturbed arg-max are evaluated in
+ *   double; weights are rounded to float on output. */
+int specs_subsample(specs_ctx* ctx, const float* blk_lp_target, const float* blk_lp_gen,
+                    const float* reward, const int32_t* cand_offsets, int32_t P, float beta,
+                    const float* uniforms, int32_t* chosen, float* weights,
+                    float tau, uint8_t* accept, void* cuda_stream);
+
+/* Same as specs_subsample with the block log-probabilities given in double
+ * (the unrounded sums from specs_score_blocks / specs_block_sums). */
+int specs_subsample_f64(specs_ctx* ctx, const double* blk_lp_target, const double* blk_lp_gen,
+                        const float* reward, const int32_t* cand_offsets, int32_t P, float beta,
+                        const float* uniforms, int32_t* chosen, float* weights,
+                        float tau, uint8_t* accept, void* cuda_stream);
+
+/* The dynamic-switching test alone (Algorithm 1, Step III; Section 2.3):
+ * accept[p] = 1 iff the largest reward among ALL candidates of problem p is
+ * strictly above tau, i.e. the draft model may generate the next step.  The call
+ * is a stateless predicate; whether a switch is permanent is the caller's policy. */
+int specs_accept(specs_ctx* ctx, const float* reward, const int32_t* cand_offsets, int32_t P,
+                 float tau, uint8_t* accept, void* cuda_stream);
+
+/* Synchronise `cuda_stream`, return the device status word (a combination of
+ * SPECS_DEV_* bits, 0 if clean) through *h_bits and clear it.  Returns
+ * SPECS_ERR_DEVICE_TIMEOUT / SPECS_ERR_TOKEN_RANGE (timeout first) when a bit is
+ * set, SPECS_OK otherwise.  h_bits may be NULL. */
+int specs_device_status(specs_ctx* ctx, uint32_t* h_bits, void* cuda_stream);
+
+/* One whole beam step from HOST buffers (the end-to-end path): copies the step's
+ * inputs to the device, runs specs_score_blocks, specs_block_sums on the
+ * generator's per-token log-probabilities, and specs_subsample_f64 with the switch
+ * test, copies the results back and synchronises the stream before returning.
+ * W_vocab is the model's weight and stays a DEVICE pointer.  The context keeps
+ * grow-only device and pinned staging buffers for this call, so it may allocate on
+ * first use or when sizes grow.  h_block_offsets and h_cand_offsets are validated
+ * (SPECS_ERR_OFFSETS).  h_gen_tok_logprob == NULL means pi_gen = pi_target.
+ * Any output pointer except h_chosen may be NULL. */
+int specs_beam_step_host(specs_ctx* ctx,
+                         const void* h_hidden, const void* W_vocab, const int32_t* h_token_ids,
+                         const int64_t* h_block_offsets, const int32_t* h_cand_offsets,
+                         const float* h_gen_tok_logprob, const float* h_reward, const float* h_uniforms,
+                         int64_t rows, int32_t d, int32_t V, int32_t B, int32_t P,
+                         float beta, float tau,
+                         float* h_tok_logprob, double* h_blk_logprob, float* h_weights,
+                         int32_t* h_chosen, uint8_t* h_accept, void* cuda_stream);
+
+/* Per-launch timing of the tensor-core scoring kernel.  specs_set_timing(ctx, 1)
+ * makes every later specs_score_blocks call on this context record a CUDA event
+ * before and after that kernel on the call's own stream (a few microseconds each;
+ * off by default) and forgets earlier records; specs_set_timing(ctx, 0) stops.
+ * specs_score_kernel_ms() waits for the recorded launches, returns their MEAN
+ * duration in milliseconds, stores their number in *h_launches (may be NULL) and
+ * forgets them; it returns a negative value when nothing was recorded. */
+int   specs_set_timing(specs_ctx* ctx, int enabled);
+float specs_score_kernel_ms(specs_ctx* ctx, int32_t* h_launches);
+
+/* The work-unit plan of the tensor-core scoring kernel, for inspection and tests
+ * (pure host arithmetic, needs no device).  The row tiles (128 rows) x vocabulary
+ * tiles (256 entries) grid is processed in waves; in a wave, gm row tiles are live
+ * and the vocabulary is cut into s contiguous chunks, one persistent CTA per
+ * (row tile, chunk).  h_out12 receives: row_tiles, vocab_tiles, k_blocks, grid,
+ * group_m, split_full, full_waves, rem_m, split_rem, waves, and the workspace size
+ * in bytes as two 31-bit halves (low, high). */
+int specs_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t* h_out12);
+
+/* Work unit of CTA `cta` in wave `wave` under that plan: h_out3 = {row tile,
+ * first vocab tile, one-past-last vocab tile}; row tile -1 when the CTA idles. */
+int specs_score_plan_unit(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t wave, int32_t cta,
+                          int32_t* h_out3);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECS_H_ */

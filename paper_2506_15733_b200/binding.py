@@ -1,0 +1,221 @@
+"""Thin ctypes binding over the C ABI declared in ``include/specs.h``.
+
+Argument marshalling only: every step of the method runs in the CUDA kernels of
+the shared library.  Device buffers are torch tensors (torch is used for device
+memory and streams, nothing else); functions take ``tensor.data_ptr()`` and the
+current torch stream.  If the shared library is missing the first call raises --
+there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libspecs_b200.so")
+_lib = None
+
+OK = 0
+ENGINE_TCGEN05 = 0
+ENGINE_SIMT = 1
+DEV_TIMEOUT = 0x1
+DEV_TOKEN_RANGE = 0x2
+
+_vp, _i32, _i64, _f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
+
+# name -> (restype, argtypes); mirrors include/specs.h one to one
+SIGNATURES = {
+    "specs_status_string": (C.c_char_p, [C.c_int]),
+    "specs_create": (C.c_int, [C.POINTER(_vp), C.c_int]),
+    "specs_destroy": (C.c_int, [_vp]),
+    "specs_set_engine": (C.c_int, [_vp, C.c_int]),
+    "specs_sm_count": (C.c_int, [_vp]),
+    "specs_score_workspace_bytes": (C.c_size_t, [_vp, _i64, _i32, _i32]),
+    "specs_score_blocks": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp,
+                                     C.c_size_t, _vp]),
+    "specs_block_sums": (C.c_int, [_vp, _vp, _vp, _i32, _vp, _vp, _vp]),
+    "specs_subsample": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _f32, _vp, _vp, _vp, _f32, _vp, _vp]),
+    "specs_subsample_f64": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _f32, _vp, _vp, _vp, _f32, _vp, _vp]),
+    "specs_accept": (C.c_int, [_vp, _vp, _vp, _i32, _f32, _vp, _vp]),
+    "specs_device_status": (C.c_int, [_vp, C.POINTER(C.c_uint32), _vp]),
+    "specs_beam_step_host": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32,
+                                       _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "specs_set_timing": (C.c_int, [_vp, C.c_int]),
+    "specs_score_kernel_ms": (C.c_float, [_vp, C.POINTER(_i32)]),
+    "specs_score_plan": (C.c_int, [_i64, _i32, _i32, _i32, C.POINTER(_i32)]),
+    "specs_score_plan_unit": (C.c_int, [_i64, _i32, _i32, _i32, _i32, _i32, C.POINTER(_i32)]),
+}
+
+
+class SpecsError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({status_string(status)})")
+
+
+def load_library():
+    """Load the shared library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2506_15733_b200.build` "
+            "(there is no fallback implementation)")
+    lib = C.CDLL(_LIB_PATH)
+    for name, (res, args) in SIGNATURES.items():
+        fn = getattr(lib, name)
+        fn.restype, fn.argtypes = res, args
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load_library().specs_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise SpecsError(status, where)
+
+
+def _ptr(t) -> Optional[int]:
+    """Device (or host) address of a torch tensor / numpy array, None for None."""
+    if t is None:
+        return None
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return t.data_ptr()
+
+
+def _stream() -> Optional[int]:
+    import torch
+    return torch.cuda.current_stream().cuda_stream or None
+
+
+def score_plan(rows: int, d: int, V: int, num_sms: int) -> dict:
+    out = (_i32 * 12)()
+    _check(load_library().specs_score_plan(rows, d, V, num_sms, out), "specs_score_plan")
+    keys = ["row_tiles", "vocab_tiles", "k_blocks", "grid", "group_m", "split_full", "full_waves", "rem_m",
+            "split_rem", "waves"]
+    plan = {k: int(out[i]) for i, k in enumerate(keys)}
+    plan["workspace_bytes"] = int(out[10]) + (int(out[11]) << 31)
+    return plan
+
+
+def score_plan_unit(rows: int, d: int, V: int, num_sms: int, wave: int, cta: int):
+    out = (_i32 * 3)()
+    _check(load_library().specs_score_plan_unit(rows, d, V, num_sms, wave, cta, out), "specs_score_plan_unit")
+    return int(out[0]), int(out[1]), int(out[2])
+
+
+class Context:
+    """Owns a ``specs_ctx`` on one CUDA device."""
+
+    def __init__(self, device: int = 0):
+        self._lib = load_library()
+        h = _vp()
+        _check(self._lib.specs_create(C.byref(h), int(device)), "specs_create")
+        self._h = h
+        self.device = int(device)
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.specs_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- small accessors
+    def set_engine(self, engine: int):
+        _check(self._lib.specs_set_engine(self._h, int(engine)), "specs_set_engine")
+
+    def sm_count(self) -> int:
+        return int(self._lib.specs_sm_count(self._h))
+
+    def score_workspace_bytes(self, rows: int, d: int, V: int) -> int:
+        return int(self._lib.specs_score_workspace_bytes(self._h, rows, d, V))
+
+    def set_timing(self, enabled: bool):
+        _check(self._lib.specs_set_timing(self._h, 1 if enabled else 0), "specs_set_timing")
+
+    def score_kernel_ms(self):
+        n = _i32(0)
+        ms = float(self._lib.specs_score_kernel_ms(self._h, C.byref(n)))
+        return ms, int(n.value)
+
+    def device_status(self, raise_on_error: bool = False) -> int:
+        bits = C.c_uint32(0)
+        st = self._lib.specs_device_status(self._h, C.byref(bits), _stream())
+        if raise_on_error:
+            _check(st, "specs_device_status")
+        return int(bits.value)
+
+    # -- the calls of the path (same names as the C ABI)
+    def specs_score_blocks(self, hidden, w_vocab, token_ids, block_offsets, tok_logprob,
+                           blk_logprob=None, blk_logprob_f64=None, workspace=None):
+        rows, d = hidden.shape
+        V = w_vocab.shape[0]
+        B = block_offsets.shape[0] - 1
+        ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+        _check(self._lib.specs_score_blocks(self._h, _ptr(hidden), _ptr(w_vocab), _ptr(token_ids),
+                                            _ptr(block_offsets), rows, d, V, B, _ptr(tok_logprob),
+                                            _ptr(blk_logprob), _ptr(blk_logprob_f64), _ptr(workspace), ws_bytes,
+                                            _stream()), "specs_score_blocks")
+
+    def specs_block_sums(self, per_token, block_offsets, out=None, out_f64=None):
+        B = block_offsets.shape[0] - 1
+        _check(self._lib.specs_block_sums(self._h, _ptr(per_token), _ptr(block_offsets), B, _ptr(out),
+                                          _ptr(out_f64), _stream()), "specs_block_sums")
+
+    def specs_subsample(self, blk_lp_target, blk_lp_gen, reward, cand_offsets, beta, uniforms, chosen,
+                        weights=None, tau=float("nan"), accept=None):
+        import torch
+        P = cand_offsets.shape[0] - 1
+        f64 = blk_lp_target is not None and blk_lp_target.dtype == torch.float64
+        if blk_lp_gen is not None and (blk_lp_gen.dtype == torch.float64) != f64:
+            raise TypeError("target and generator block log-probs must have the same dtype")
+        fn = self._lib.specs_subsample_f64 if f64 else self._lib.specs_subsample
+        _check(fn(self._h, _ptr(blk_lp_target), _ptr(blk_lp_gen), _ptr(reward), _ptr(cand_offsets), P, float(beta),
+                  _ptr(uniforms), _ptr(chosen), _ptr(weights), float(tau), _ptr(accept), _stream()),
+               "specs_subsample")
+
+    def specs_accept(self, reward, cand_offsets, tau, accept):
+        P = cand_offsets.shape[0] - 1
+        _check(self._lib.specs_accept(self._h, _ptr(reward), _ptr(cand_offsets), P, float(tau), _ptr(accept),
+                                      _stream()), "specs_accept")
+
+    def specs_beam_step_host(self, h_hidden, w_vocab, h_token_ids, h_block_offsets, h_cand_offsets,
+                             h_gen_tok_logprob, h_reward, h_uniforms, beta, tau,
+                             h_tok_logprob, h_blk_logprob, h_weights, h_chosen, h_accept):
+        """Host tensors/arrays in, host tensors/arrays out; ``w_vocab`` is a device tensor."""
+        rows, d = h_hidden.shape
+        V = w_vocab.shape[0]
+        B = h_block_offsets.shape[0] - 1
+        P = h_cand_offsets.shape[0] - 1
+        _check(self._lib.specs_beam_step_host(
+            self._h, _ptr(h_hidden), _ptr(w_vocab), _ptr(h_token_ids), _ptr(h_block_offsets), _ptr(h_cand_offsets),
+            _ptr(h_gen_tok_logprob), _ptr(h_reward), _ptr(h_uniforms), rows, d, V, B, P, float(beta), float(tau),
+            _ptr(h_tok_logprob), _ptr(h_blk_logprob), _ptr(h_weights), _ptr(h_chosen), _ptr(h_accept), _stream()),
+            "specs_beam_step_host")
+
+
+# ---------------------------------------------------------------------------- torch helpers (marshalling only)
+
+def bf16_bits_to_device(bits: np.ndarray, device="cuda"):
+    """uint16 bf16 bit patterns (numpy) -> torch.bfloat16 tensor on the device, bit for bit."""
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16))
+    return t.to(device).view(torch.bfloat16)
+
+
+def bf16_bits_to_pinned(bits: np.ndarray):
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).pin_memory()
+    return t.view(torch.bfloat16)

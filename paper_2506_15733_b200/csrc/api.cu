@@ -1,0 +1,397 @@
+// C ABI of the library: argument validation, the work-unit planner, context management and
+// the host-buffer convenience entry point.  All arithmetic of the method runs in the kernels
+// of the other translation units.
+#include <cstring>
+#include <new>
+
+#include "specs_internal.h"
+
+namespace specs {
+
+// ---------------------------------------------------------------------------------- planner
+ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms) {
+    ScorePlan p;
+    std::memset(&p, 0, sizeof(p));
+    p.rows = rows; p.d = d; p.V = V;
+    p.row_tiles = (int32_t)((rows + kBlockM - 1) / kBlockM);
+    p.vocab_tiles = (V + kBlockN - 1) / kBlockN;
+    p.k_blocks = (d + kBlockK - 1) / kBlockK;
+    p.grid = num_sms;
+    if (p.row_tiles == 0) return p;
+
+    // Full waves: the fewest vocabulary chunks s (hence the most row tiles gm = grid / s sharing
+    // each streamed W tile) such that the wave's hidden tiles stay well inside L2 and at most 2%
+    // of the CTAs idle.
+    const double tile_bytes = (double)kBlockM * d * 2.0;
+    const double l2_budget = 50.0e6;
+    int best_s = num_sms;                     // gm = 1 always fits
+    for (int s = 1; s <= num_sms; ++s) {
+        const int gm = num_sms / s;
+        if (gm * tile_bytes > l2_budget && gm > 1) continue;
+        if ((double)(gm * s) < 0.98 * num_sms) continue;
+        best_s = s;
+        break;
+    }
+    if (best_s > p.vocab_tiles) best_s = p.vocab_tiles;       // a chunk holds at least one vocab tile
+    p.split_full = best_s;
+    p.group_m = num_sms / best_s;
+    p.full_waves = p.row_tiles / p.group_m;
+    p.rem_m = p.row_tiles - p.full_waves * p.group_m;
+    if (p.rem_m > 0) {
+        int s = num_sms / p.rem_m;
+        if (s > p.vocab_tiles) s = p.vocab_tiles;
+        if (s < 1) s = 1;
+        p.split_rem = s;
+    }
+    p.waves = p.full_waves + (p.rem_m > 0 ? 1 : 0);
+    return p;
+}
+
+size_t plan_workspace_bytes(const ScorePlan& p) {
+    const size_t slots = (size_t)(p.waves > 0 ? p.waves : 1) * (size_t)p.grid;
+    return slots * kTripleFloats * sizeof(float);
+}
+
+}  // namespace specs
+
+using namespace specs;
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_offsets64(const int64_t* off, int64_t count, int64_t total) {
+    if (off[0] != 0) return SPECS_ERR_OFFSETS;
+    for (int64_t i = 0; i < count; ++i)
+        if (off[i + 1] < off[i]) return SPECS_ERR_OFFSETS;
+    return off[count] == total ? SPECS_OK : SPECS_ERR_OFFSETS;
+}
+int check_offsets32(const int32_t* off, int64_t count, int64_t total) {
+    if (off[0] != 0) return SPECS_ERR_OFFSETS;
+    for (int64_t i = 0; i < count; ++i)
+        if (off[i + 1] < off[i]) return SPECS_ERR_OFFSETS;
+    return off[count] == total ? SPECS_OK : SPECS_ERR_OFFSETS;
+}
+
+int check_score_shapes(int64_t rows, int32_t d, int32_t V, int32_t B) {
+    if (rows < 0 || d <= 0 || (d % 8) != 0 || V <= 0 || B < 0) return SPECS_ERR_SHAPE;
+    if (rows > (int64_t)1 << 31) return SPECS_ERR_LIMIT;
+    return SPECS_OK;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        if (prev == dev) prev = -1;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+}  // namespace
+
+extern "C" {
+
+const char* specs_status_string(int status) {
+    switch (status) {
+        case SPECS_OK: return "ok";
+        case SPECS_ERR_NULL: return "a required pointer is NULL";
+        case SPECS_ERR_SHAPE: return "invalid shape (negative size, d not a positive multiple of 8, ...)";
+        case SPECS_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case SPECS_ERR_WORKSPACE: return "workspace too small";
+        case SPECS_ERR_OFFSETS: return "offsets must start at 0, be non-decreasing and end at the total";
+        case SPECS_ERR_ARCH: return "device is not an sm_100-class GPU";
+        case SPECS_ERR_CUDA: return "a CUDA call failed";
+        case SPECS_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel expired";
+        case SPECS_ERR_TOKEN_RANGE: return "a drafted token id was outside [0, V)";
+        case SPECS_ERR_LIMIT: return "a size exceeds a documented maximum";
+        default: return "unknown status";
+    }
+}
+
+int specs_create(specs_ctx** out, int device) {
+    if (!out) return SPECS_ERR_NULL;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+        cudaGetLastError();
+        return SPECS_ERR_CUDA;
+    }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return SPECS_ERR_CUDA;
+    if (prop.major != 10) return SPECS_ERR_ARCH;
+    DeviceGuard guard(device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+
+    specs_ctx* ctx = new (std::nothrow) specs_ctx();
+    if (!ctx) return SPECS_ERR_CUDA;
+    ctx->device = device;
+    ctx->num_sms = prop.multiProcessorCount;
+
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+        delete ctx;
+        return SPECS_ERR_CUDA;
+    }
+    ctx->encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    if (cudaMalloc(&ctx->d_status, sizeof(uint32_t)) != cudaSuccess ||
+        cudaMemset(ctx->d_status, 0, sizeof(uint32_t)) != cudaSuccess) {
+        if (ctx->d_status) cudaFree(ctx->d_status);
+        delete ctx;
+        return SPECS_ERR_CUDA;
+    }
+    *out = ctx;
+    return SPECS_OK;
+}
+
+int specs_destroy(specs_ctx* ctx) {
+    if (!ctx) return SPECS_OK;
+    DeviceGuard guard(ctx->device);
+    for (auto& t : ctx->timed) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
+    if (ctx->arena) cudaFree(ctx->arena);
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    delete ctx;
+    return SPECS_OK;
+}
+
+int specs_set_engine(specs_ctx* ctx, int engine) {
+    if (!ctx) return SPECS_ERR_NULL;
+    if (engine != SPECS_ENGINE_TCGEN05 && engine != SPECS_ENGINE_SIMT) return SPECS_ERR_SHAPE;
+    ctx->engine = engine;
+    return SPECS_OK;
+}
+
+int specs_sm_count(const specs_ctx* ctx) { return ctx ? ctx->num_sms : 0; }
+
+size_t specs_score_workspace_bytes(const specs_ctx* ctx, int64_t rows, int32_t d, int32_t V) {
+    if (!ctx || check_score_shapes(rows, d, V, 0) != SPECS_OK) return 0;
+    return plan_workspace_bytes(make_score_plan(rows, d, V, ctx->num_sms));
+}
+
+int specs_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t* h_out12) {
+    if (!h_out12) return SPECS_ERR_NULL;
+    if (check_score_shapes(rows, d, V, 0) != SPECS_OK || num_sms <= 0) return SPECS_ERR_SHAPE;
+    const ScorePlan p = make_score_plan(rows, d, V, num_sms);
+    const int32_t v[12] = {p.row_tiles, p.vocab_tiles, p.k_blocks, p.grid, p.group_m, p.split_full,
+                           p.full_waves, p.rem_m, p.split_rem, p.waves,
+                           (int32_t)(plan_workspace_bytes(p) & 0x7fffffff), (int32_t)(plan_workspace_bytes(p) >> 31)};
+    std::memcpy(h_out12, v, sizeof(v));
+    return SPECS_OK;
+}
+
+int specs_score_plan_unit(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t wave, int32_t cta,
+                          int32_t* h_out3) {
+    if (!h_out3) return SPECS_ERR_NULL;
+    if (check_score_shapes(rows, d, V, 0) != SPECS_OK || num_sms <= 0) return SPECS_ERR_SHAPE;
+    const ScorePlan p = make_score_plan(rows, d, V, num_sms);
+    int mt = -1, nb = 0, ne = 0;
+    if (wave < 0 || wave >= p.waves || cta < 0 || cta >= p.grid || !plan_unit(p, wave, cta, &mt, &nb, &ne)) {
+        h_out3[0] = -1; h_out3[1] = 0; h_out3[2] = 0;
+        return SPECS_OK;
+    }
+    h_out3[0] = mt; h_out3[1] = nb; h_out3[2] = ne;
+    return SPECS_OK;
+}
+
+int specs_score_blocks(specs_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* token_ids,
+                       const int64_t* block_offsets, int64_t rows, int32_t d, int32_t V, int32_t B,
+                       float* tok_logprob, float* blk_logprob, double* blk_logprob_f64, void* workspace,
+                       size_t workspace_bytes, void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    int st = check_score_shapes(rows, d, V, B);
+    if (st != SPECS_OK) return st;
+    if (!W_vocab || (B > 0 && !block_offsets)) return SPECS_ERR_NULL;
+    if (rows > 0 && (!hidden || !token_ids || !tok_logprob)) return SPECS_ERR_NULL;
+    if (!aligned16(hidden) || !aligned16(W_vocab) || !aligned16(workspace)) return SPECS_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+
+    if (rows > 0) {
+        if (ctx->engine == SPECS_ENGINE_SIMT) {
+            st = launch_score_simt(ctx, hidden, W_vocab, token_ids, rows, d, V, tok_logprob, stream);
+            if (st != SPECS_OK) return st;
+        } else {
+            const ScorePlan plan = make_score_plan(rows, d, V, ctx->num_sms);
+            if (!workspace) return SPECS_ERR_NULL;
+            if (workspace_bytes < plan_workspace_bytes(plan)) return SPECS_ERR_WORKSPACE;
+            st = launch_score_tcgen05(ctx, plan, hidden, W_vocab, token_ids, static_cast<float*>(workspace), stream);
+            if (st != SPECS_OK) return st;
+            st = launch_merge(ctx, plan, static_cast<const float*>(workspace), token_ids, tok_logprob, stream);
+            if (st != SPECS_OK) return st;
+        }
+    }
+    if (B > 0 && (blk_logprob || blk_logprob_f64))
+        return launch_block_sums(tok_logprob, block_offsets, B, blk_logprob, blk_logprob_f64, stream);
+    return SPECS_OK;
+}
+
+int specs_block_sums(specs_ctx* ctx, const float* per_token, const int64_t* block_offsets, int32_t B, float* out,
+                     double* out_f64, void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    if (B < 0) return SPECS_ERR_SHAPE;
+    if (B == 0) return SPECS_OK;
+    if (!block_offsets || (!out && !out_f64)) return SPECS_ERR_NULL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+    return launch_block_sums(per_token, block_offsets, B, out, out_f64, static_cast<cudaStream_t>(cuda_stream));
+}
+
+static int subsample_common(specs_ctx* ctx, const void* lp_t, const void* lp_g, bool f64, const float* reward,
+                            const int32_t* cand_offsets, int32_t P, float beta, const float* uniforms,
+                            int32_t* chosen, float* weights, float tau, uint8_t* accept, void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    if (P < 0) return SPECS_ERR_SHAPE;
+    if (P == 0) return SPECS_OK;
+    if (!reward || !cand_offsets || !uniforms || !chosen) return SPECS_ERR_NULL;
+    if (lp_g && !lp_t) return SPECS_ERR_NULL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+    return launch_subsample(lp_t, lp_g, f64, reward, cand_offsets, P, beta, uniforms, chosen, weights, tau, accept,
+                            static_cast<cudaStream_t>(cuda_stream));
+}
+
+int specs_subsample(specs_ctx* ctx, const float* blk_lp_target, const float* blk_lp_gen, const float* reward,
+                    const int32_t* cand_offsets, int32_t P, float beta, const float* uniforms, int32_t* chosen,
+                    float* weights, float tau, uint8_t* accept, void* cuda_stream) {
+    return subsample_common(ctx, blk_lp_target, blk_lp_gen, false, reward, cand_offsets, P, beta, uniforms, chosen,
+                            weights, tau, accept, cuda_stream);
+}
+
+int specs_subsample_f64(specs_ctx* ctx, const double* blk_lp_target, const double* blk_lp_gen, const float* reward,
+                        const int32_t* cand_offsets, int32_t P, float beta, const float* uniforms, int32_t* chosen,
+                        float* weights, float tau, uint8_t* accept, void* cuda_stream) {
+    return subsample_common(ctx, blk_lp_target, blk_lp_gen, true, reward, cand_offsets, P, beta, uniforms, chosen,
+                            weights, tau, accept, cuda_stream);
+}
+
+int specs_accept(specs_ctx* ctx, const float* reward, const int32_t* cand_offsets, int32_t P, float tau,
+                 uint8_t* accept, void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    if (P < 0) return SPECS_ERR_SHAPE;
+    if (P == 0) return SPECS_OK;
+    if (!reward || !cand_offsets || !accept) return SPECS_ERR_NULL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+    return launch_accept(reward, cand_offsets, P, tau, accept, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int specs_device_status(specs_ctx* ctx, uint32_t* h_bits, void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint32_t bits = 0;
+    if (cudaMemcpyAsync(&bits, ctx->d_status, sizeof(bits), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaMemsetAsync(ctx->d_status, 0, sizeof(bits), stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess)
+        return SPECS_ERR_CUDA;
+    if (h_bits) *h_bits = bits;
+    if (bits & SPECS_DEV_TIMEOUT) return SPECS_ERR_DEVICE_TIMEOUT;
+    if (bits & SPECS_DEV_TOKEN_RANGE) return SPECS_ERR_TOKEN_RANGE;
+    return SPECS_OK;
+}
+
+int specs_set_timing(specs_ctx* ctx, int enabled) {
+    if (!ctx) return SPECS_ERR_NULL;
+    ctx->timing = enabled != 0;
+    ctx->timed_used = 0;
+    return SPECS_OK;
+}
+
+float specs_score_kernel_ms(specs_ctx* ctx, int32_t* h_launches) {
+    if (h_launches) *h_launches = 0;
+    if (!ctx || ctx->timed_used == 0) return -1.0f;
+    DeviceGuard guard(ctx->device);
+    double total = 0.0;
+    for (size_t i = 0; i < ctx->timed_used; ++i) {
+        float ms = 0.0f;
+        if (cudaEventSynchronize(ctx->timed[i].stop) != cudaSuccess ||
+            cudaEventElapsedTime(&ms, ctx->timed[i].start, ctx->timed[i].stop) != cudaSuccess)
+            return -1.0f;
+        total += ms;
+    }
+    if (h_launches) *h_launches = (int32_t)ctx->timed_used;
+    const float mean = (float)(total / (double)ctx->timed_used);
+    ctx->timed_used = 0;
+    return mean;
+}
+
+int specs_beam_step_host(specs_ctx* ctx, const void* h_hidden, const void* W_vocab, const int32_t* h_token_ids,
+                         const int64_t* h_block_offsets, const int32_t* h_cand_offsets,
+                         const float* h_gen_tok_logprob, const float* h_reward, const float* h_uniforms,
+                         int64_t rows, int32_t d, int32_t V, int32_t B, int32_t P, float beta, float tau,
+                         float* h_tok_logprob, double* h_blk_logprob, float* h_weights, int32_t* h_chosen,
+                         uint8_t* h_accept, void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    int st = check_score_shapes(rows, d, V, B);
+    if (st != SPECS_OK) return st;
+    if (P < 0) return SPECS_ERR_SHAPE;
+    if (!W_vocab || !h_block_offsets || !h_cand_offsets || !h_chosen) return SPECS_ERR_NULL;
+    if (rows > 0 && (!h_hidden || !h_token_ids)) return SPECS_ERR_NULL;
+    if (B > 0 && (!h_reward || !h_uniforms)) return SPECS_ERR_NULL;
+    if (!aligned16(W_vocab)) return SPECS_ERR_ALIGN;
+    if ((st = check_offsets64(h_block_offsets, B, rows)) != SPECS_OK) return st;
+    if ((st = check_offsets32(h_cand_offsets, P, B)) != SPECS_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+
+    const ScorePlan plan = make_score_plan(rows, d, V, ctx->num_sms);
+    // carve the arena (every piece 256-byte aligned)
+    size_t off = 0;
+    auto carve = [&off](size_t bytes) { const size_t at = off; off += (bytes + 255) & ~(size_t)255; return at; };
+    const size_t o_hidden = carve((size_t)rows * d * 2), o_ids = carve((size_t)rows * 4);
+    const size_t o_boff = carve((size_t)(B + 1) * 8), o_coff = carve((size_t)(P + 1) * 4);
+    const size_t o_gen = carve((size_t)rows * 4), o_rew = carve((size_t)B * 4), o_uni = carve((size_t)B * 4);
+    const size_t o_tok = carve((size_t)rows * 4), o_blk_t = carve((size_t)B * 8), o_blk_g = carve((size_t)B * 8);
+    const size_t o_wts = carve((size_t)B * 4), o_cho = carve((size_t)P * 4), o_acc = carve((size_t)P);
+    const size_t ws_bytes = plan_workspace_bytes(plan);
+    const size_t o_ws = carve(ws_bytes);
+    if (off > ctx->arena_bytes) {
+        if (ctx->arena) { cudaStreamSynchronize(stream); cudaFree(ctx->arena); ctx->arena = nullptr; ctx->arena_bytes = 0; }
+        if (cudaMalloc(&ctx->arena, off) != cudaSuccess) return SPECS_ERR_CUDA;
+        ctx->arena_bytes = off;
+    }
+    uint8_t* A = static_cast<uint8_t*>(ctx->arena);
+    auto h2d = [&](size_t at, const void* src, size_t bytes) {
+        return bytes == 0 || cudaMemcpyAsync(A + at, src, bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    };
+    auto d2h = [&](void* dst, size_t at, size_t bytes) {
+        return !dst || bytes == 0 || cudaMemcpyAsync(dst, A + at, bytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    };
+    bool ok = h2d(o_hidden, h_hidden, (size_t)rows * d * 2) && h2d(o_ids, h_token_ids, (size_t)rows * 4) &&
+              h2d(o_boff, h_block_offsets, (size_t)(B + 1) * 8) && h2d(o_coff, h_cand_offsets, (size_t)(P + 1) * 4) &&
+              h2d(o_rew, h_reward, (size_t)B * 4) && h2d(o_uni, h_uniforms, (size_t)B * 4);
+    if (ok && h_gen_tok_logprob) ok = h2d(o_gen, h_gen_tok_logprob, (size_t)rows * 4);
+    if (!ok) return SPECS_ERR_CUDA;
+
+    st = specs_score_blocks(ctx, A + o_hidden, W_vocab, reinterpret_cast<int32_t*>(A + o_ids),
+                            reinterpret_cast<int64_t*>(A + o_boff), rows, d, V, B,
+                            reinterpret_cast<float*>(A + o_tok), nullptr, reinterpret_cast<double*>(A + o_blk_t),
+                            A + o_ws, ws_bytes, cuda_stream);
+    if (st != SPECS_OK) return st;
+    const double* gen_blk = nullptr;
+    if (h_gen_tok_logprob) {
+        st = specs_block_sums(ctx, reinterpret_cast<float*>(A + o_gen), reinterpret_cast<int64_t*>(A + o_boff), B,
+                              nullptr, reinterpret_cast<double*>(A + o_blk_g), cuda_stream);
+        if (st != SPECS_OK) return st;
+        gen_blk = reinterpret_cast<double*>(A + o_blk_g);
+    }
+    st = specs_subsample_f64(ctx, reinterpret_cast<double*>(A + o_blk_t), gen_blk, reinterpret_cast<float*>(A + o_rew),
+                             reinterpret_cast<int32_t*>(A + o_coff), P, beta, reinterpret_cast<float*>(A + o_uni),
+                             reinterpret_cast<int32_t*>(A + o_cho), reinterpret_cast<float*>(A + o_wts), tau,
+                             reinterpret_cast<uint8_t*>(A + o_acc), cuda_stream);
+    if (st != SPECS_OK) return st;
+    ok = d2h(h_tok_logprob, o_tok, (size_t)rows * 4) && d2h(h_blk_logprob, o_blk_t, (size_t)B * 8) &&
+         d2h(h_weights, o_wts, (size_t)B * 4) && d2h(h_chosen, o_cho, (size_t)P * 4) &&
+         d2h(h_accept, o_acc, (size_t)P);
+    if (!ok || cudaStreamSynchronize(stream) != cudaSuccess) return SPECS_ERR_CUDA;
+    return SPECS_OK;
+}
+
+}  // extern "C"

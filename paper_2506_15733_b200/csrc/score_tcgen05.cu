@@ -1,0 +1,404 @@
+// LM-head scoring kernel for sm_100a: hidden[rows,d] x W_vocab[V,d]^T on the 5th-generation
+// tensor cores with a fused online log-sum-exp + drafted-logit gather epilogue.  The rows x V
+// logits live only in tensor memory (TMEM); what reaches HBM is one (max, sum-exp, logit)
+// triple per row and per vocabulary chunk.
+//
+// This is the "computing logits of each token" step of scoring a drafted block with the
+// target model (Section 2 of the paper; Appendix E.3 restricts it to the new block's tokens).
+//
+// One persistent CTA per SM, 192 threads, three roles:
+//   warp 0      TMA producer: cp.async.bulk.tensor loads of a 128x64 hidden tile and a 256x64
+//               W tile per k-block into a 4-stage, 128-byte-swizzled shared-memory ring.
+//   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32);
+//               the accumulator is one of two 128-lane x 256-column TMEM buffers, so the
+//               epilogue of vocabulary tile j overlaps the MMAs of tile j+1.
+//   warps 2-5   epilogue: thread = one row (TMEM lane).  tcgen05.ld 32 columns at a time,
+//               running max / rescaled sum of 2^x / select of the drafted id's logit, all in
+//               registers across the CTA's run of vocabulary tiles.
+// Every mbarrier wait is bounded; on expiry the CTA raises SPECS_DEV_TIMEOUT, all roles leave
+// their loops, the producer waits (bounded) for its copies in flight, TMEM is freed and the
+// kernel returns.
+#include <cuda_bf16.h>
+
+#include "specs_internal.h"
+
+namespace specs {
+namespace {
+
+constexpr int kStages = 4;
+constexpr int kUmmaK = 16;
+constexpr uint32_t kABytes = kBlockM * kBlockK * 2;      // 16 KB
+constexpr uint32_t kBBytes = kBlockN * kBlockK * 2;      // 32 KB
+constexpr uint32_t kStageBytes = kABytes + kBBytes;      // 48 KB
+constexpr int kThreads = 192;
+constexpr int kEpilogueThreads = 128;
+constexpr uint32_t kTmemCols = 512;                      // two 256-column accumulators
+constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kStages * kStageBytes + 256 /*barriers*/;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
+constexpr unsigned long long kDrainLimitNs = 20000000ull;    // 20 ms per stage when draining after an abort
+constexpr float kLog2e = 1.4426950408889634f;
+
+// ---- thin PTX wrappers -------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false if the CTA-wide abort flag is (or becomes) set.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          unsigned long long limit_ns, bool raise) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    uint32_t spins = 0;
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 0xFFu) == 0u) {
+            if (raise && *abort_flag) return false;
+            if (global_timer_ns() - t0 > limit_ns) {
+                if (raise) *abort_flag = 1u;
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c_inner), "r"(c_outer), "r"(bar)
+        : "memory");
+}
+// 2^x on the special-function unit (relative error about 2^-22; 2^-inf = 0).
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread i of the warp gets lane (base lane + i).
+// The load and its completion wait sit in one statement so that the registers are
+// valid as soon as the statement has executed.
+__device__ __forceinline__ void tmem_ld_32cols(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+        "tcgen05.wait::ld.sync.aligned;\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (64
+// elements) long, written by TMA with the 128-byte swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t saddr) {
+    uint64_t desc = 0;
+    desc |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);   // bits  0-13 start address / 16
+    desc |= static_cast<uint64_t>(1) << 16;                   // bits 16-29 leading byte offset (unused here)
+    desc |= static_cast<uint64_t>(1024 >> 4) << 32;           // bits 32-45 stride byte offset / 16
+    desc |= static_cast<uint64_t>(1) << 46;                   // bits 46-47 descriptor version (sm_100)
+    desc |= static_cast<uint64_t>(2) << 61;                   // bits 61-63 swizzle mode: 128 bytes
+    return desc;
+}
+// Instruction descriptor: dense, fp32 accumulate, A and B bf16, both K-major, M x N.
+__host__ __device__ constexpr uint32_t instr_desc_bf16(int m, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
+           (static_cast<uint32_t>(m >> 4) << 24);
+}
+
+struct SharedLayout {
+    uint64_t full[kStages];      // TMA -> MMA: stage holds data
+    uint64_t empty[kStages];     // MMA -> TMA: stage may be overwritten
+    uint64_t acc_full[2];        // MMA -> epilogue: accumulator complete
+    uint64_t acc_empty[2];       // epilogue -> MMA: accumulator drained
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+score_tiles_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_w,
+                   const ScorePlan plan, const int32_t* __restrict__ token_ids, float* __restrict__ workspace,
+                   uint32_t* __restrict__ status) {
+    extern __shared__ uint8_t smem_raw[];
+    // 128-byte-swizzled TMA destinations and UMMA operands must sit on 1024-byte boundaries.
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
+    uint8_t* tiles = smem_raw + pad;
+    SharedLayout* sh = reinterpret_cast<SharedLayout*>(tiles + (size_t)kStages * kStageBytes);
+    const uint32_t tiles_addr = smem_u32(tiles);
+    volatile uint32_t* abort_flag = &sh->abort_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int cta = blockIdx.x;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(&sh->full[s]), 1);
+            mbar_init(smem_u32(&sh->empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&sh->acc_full[b]), 1);
+            mbar_init(smem_u32(&sh->acc_empty[b]), kEpilogueThreads);
+        }
+        sh->abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&sh->tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&sh->tmem_base);
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            uint32_t issued = 0;
+            bool ok = true;
+            for (int w = 0; w < plan.waves && ok; ++w) {
+                int mt, nb, ne;
+                if (!plan_unit(plan, w, cta, &mt, &nb, &ne)) continue;
+                for (int n = nb; n < ne && ok; ++n) {
+                    for (int kb = 0; kb < plan.k_blocks; ++kb) {
+                        if (!mbar_wait(smem_u32(&sh->empty[stage]), phase ^ 1u, abort_flag, kWaitLimitNs, true)) {
+                            ok = false;
+                            break;
+                        }
+                        const uint32_t bar = smem_u32(&sh->full[stage]);
+                        const uint32_t a_dst = tiles_addr + stage * kStageBytes;
+                        mbar_arrive_expect_tx(bar, kStageBytes);
+                        tma_load_2d(a_dst, &map_hidden, kb * kBlockK, mt * kBlockM, bar);
+                        tma_load_2d(a_dst + kABytes, &map_w, kb * kBlockK, n * kBlockN, bar);
+                        ++issued;
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+            if (!ok) {
+                // Drain: the last min(issued, kStages) loads may still be landing in shared memory.
+                const uint32_t pending = issued < (uint32_t)kStages ? issued : (uint32_t)kStages;
+                uint32_t s = stage, ph = phase;
+                for (uint32_t i = 0; i < pending; ++i) {
+                    if (s == 0) { s = kStages - 1; ph ^= 1u; } else { --s; }
+                    mbar_wait(smem_u32(&sh->full[s]), ph, abort_flag, kDrainLimitNs, false);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_bf16(kBlockM, kBlockN);
+            uint32_t stage = 0, phase = 0;
+            uint32_t tile_count = 0;
+            bool ok = true;
+            for (int w = 0; w < plan.waves && ok; ++w) {
+                int mt, nb, ne;
+                if (!plan_unit(plan, w, cta, &mt, &nb, &ne)) continue;
+                for (int n = nb; n < ne && ok; ++n, ++tile_count) {
+                    const uint32_t buf = tile_count & 1u;
+                    const uint32_t use_phase = (tile_count >> 1) & 1u;
+                    if (!mbar_wait(smem_u32(&sh->acc_empty[buf]), use_phase ^ 1u, abort_flag, kWaitLimitNs, true)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + buf * kBlockN;
+                    for (int kb = 0; kb < plan.k_blocks; ++kb) {
+                        if (!mbar_wait(smem_u32(&sh->full[stage]), phase, abort_flag, kWaitLimitNs, true)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint32_t a_addr = tiles_addr + stage * kStageBytes;
+                        const uint64_t a_desc = smem_desc_k_major_sw128(a_addr);
+                        const uint64_t b_desc = smem_desc_k_major_sw128(a_addr + kABytes);
+#pragma unroll
+                        for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+                            // advancing 16 bf16 (32 bytes) along K inside the swizzled row: +2 in the
+                            // 16-byte units of the descriptor's start-address field
+                            tc_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                        (kb | k) != 0 ? 1u : 0u);
+                        }
+                        tc_commit(smem_u32(&sh->empty[stage]));     // frees the stage once these MMAs retire
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                    if (ok) tc_commit(smem_u32(&sh->acc_full[buf]));  // accumulator ready for the epilogue
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        const int quarter = warp & 3;                        // TMEM lanes 32*quarter .. +31 belong to this warp
+        const int row_in_tile = quarter * 32 + lane;
+        const uint32_t lane_field = static_cast<uint32_t>(quarter * 32) << 16;
+        uint32_t tile_count = 0;
+        bool ok = true;
+        for (int w = 0; w < plan.waves && ok; ++w) {
+            int mt, nb, ne;
+            if (!plan_unit(plan, w, cta, &mt, &nb, &ne)) continue;
+            const int64_t row = (int64_t)mt * kBlockM + row_in_tile;
+            const int32_t id = (row < plan.rows) ? token_ids[row] : -1;
+            // state in base-2 units: run_max = max(z) * log2(e), run_sum = sum 2^(z*log2e - run_max)
+            float run_max = -INFINITY, run_sum = 0.0f, picked = -INFINITY;
+            for (int n = nb; n < ne && ok; ++n, ++tile_count) {
+                const uint32_t buf = tile_count & 1u;
+                const uint32_t use_phase = (tile_count >> 1) & 1u;
+                if (!mbar_wait(smem_u32(&sh->acc_full[buf]), use_phase, abort_flag, kWaitLimitNs, true)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const int col_base = n * kBlockN;
+#pragma unroll 1
+                for (int c = 0; c < kBlockN / 32; ++c) {
+                    const int col0 = col_base + c * 32;
+                    const int valid = plan.V - col0;         // columns of this chunk inside the vocabulary
+                    if (valid <= 0) break;                   // uniform across the CTA
+                    float v[32];
+                    tmem_ld_32cols(tmem_base + lane_field + buf * kBlockN + c * 32, v);
+                    if (valid < 32) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = (j < valid) ? v[j] : -INFINITY;
+                    }
+                    const uint32_t rel = static_cast<uint32_t>(id - col0);
+                    if (rel < 32u) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) picked = (rel == (uint32_t)j) ? v[j] : picked;
+                    }
+                    float cmax = v[0];
+#pragma unroll
+                    for (int j = 1; j < 32; ++j) cmax = fmaxf(cmax, v[j]);
+                    const float new_max = fmaxf(run_max, cmax * kLog2e);
+                    run_sum *= ex2_approx(run_max - new_max);  // 2^-inf = 0 on the first chunk
+                    run_max = new_max;
+                    float acc0 = 0.0f, acc1 = 0.0f;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        acc0 += ex2_approx(fmaf(v[j], kLog2e, -new_max));
+                        acc1 += ex2_approx(fmaf(v[j + 1], kLog2e, -new_max));
+                    }
+                    run_sum += acc0 + acc1;
+                }
+                tc_fence_before();
+                mbar_arrive(smem_u32(&sh->acc_empty[buf]));
+            }
+            if (ok) {
+                float* slot = workspace + ((size_t)w * plan.grid + cta) * kTripleFloats;
+                slot[row_in_tile] = run_max;
+                slot[kBlockM + row_in_tile] = run_sum;
+                slot[2 * kBlockM + row_in_tile] = picked;
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && sh->abort_flag != 0u) atomicOr(status, SPECS_DEV_TIMEOUT);
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+int encode_bf16_2d(specs_ctx* ctx, CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer,
+                   uint32_t box_inner, uint32_t box_outer) {
+    const cuuint64_t dims[2] = {inner, outer};
+    const cuuint64_t strides[1] = {inner * 2};               // bytes between consecutive rows
+    const cuuint32_t box[2] = {box_inner, box_outer};
+    const cuuint32_t elem_strides[2] = {1, 1};
+    const CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+                                         strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SPECS_OK : SPECS_ERR_CUDA;
+}
+
+}  // namespace
+
+int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan, const void* hidden, const void* w_vocab,
+                         const int32_t* token_ids, float* workspace, cudaStream_t stream) {
+    static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+    CUtensorMap map_h, map_w;
+    int st = encode_bf16_2d(ctx, &map_h, hidden, (uint64_t)plan.d, (uint64_t)plan.rows, kBlockK, kBlockM);
+    if (st != SPECS_OK) return st;
+    st = encode_bf16_2d(ctx, &map_w, w_vocab, (uint64_t)plan.d, (uint64_t)plan.V, kBlockK, kBlockN);
+    if (st != SPECS_OK) return st;
+
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(score_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)kSmemBytes);
+        if (e != cudaSuccess) return SPECS_ERR_CUDA;
+        attr_set = true;
+    }
+    TimedLaunch* tl = nullptr;
+    if (ctx->timing) {
+        if (ctx->timed_used == ctx->timed.size()) {
+            TimedLaunch t;
+            if (cudaEventCreate(&t.start) != cudaSuccess || cudaEventCreate(&t.stop) != cudaSuccess)
+                return SPECS_ERR_CUDA;
+            ctx->timed.push_back(t);
+        }
+        tl = &ctx->timed[ctx->timed_used++];
+        cudaEventRecord(tl->start, stream);
+    }
+    score_tiles_kernel<<<plan.grid, kThreads, kSmemBytes, stream>>>(map_h, map_w, plan, token_ids, workspace,
+                                                                    ctx->d_status);
+    if (tl) cudaEventRecord(tl->stop, stream);
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace specs

@@ -1,0 +1,106 @@
+// Internal declarations shared by the translation units of the library.
+// Nothing here is part of the C ABI (see include/specs.h for that).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "specs.h"
+
+namespace specs {
+
+// ---- tile geometry of the tensor-core scoring kernel -----------------------------------------
+constexpr int kBlockM = 128;   // drafted rows per tile   (= TMEM lanes, one epilogue thread per row)
+constexpr int kBlockN = 256;   // vocabulary entries per tile (= fp32 TMEM columns of one accumulator)
+constexpr int kBlockK = 64;    // bf16 elements per k-block: 128 bytes, one swizzle-128B row
+constexpr int kTripleFloats = 3 * kBlockM;   // one workspace slot: max[128], sumexp[128], logit[128]
+
+// How the (row tile x vocab tile) grid is cut into persistent work units.
+//
+// Time is cut into waves.  In one wave `gm` consecutive row tiles are live and the vocabulary
+// is cut into `s` contiguous chunks, gm * s <= grid CTAs; CTA c owns row tile (c % gm) of the
+// wave and chunk (c / gm).  CTAs that share a chunk stream the same W tiles at the same pace,
+// so each W tile is fetched from HBM once per wave and hits L2 for the other row tiles, while
+// the wave's hidden-state tiles (gm * 128 * d * 2 bytes) stay L2-resident.  Every wave but the
+// last is "full" (gm = group_m, s = split_full); the last takes the remaining row tiles.
+struct ScorePlan {
+    int64_t rows;
+    int32_t d, V;
+    int32_t row_tiles;     // ceil(rows / 128)
+    int32_t vocab_tiles;   // ceil(V / 256)
+    int32_t k_blocks;      // ceil(d / 64)
+    int32_t grid;          // CTAs launched (= SM count)
+    int32_t group_m;       // row tiles per full wave
+    int32_t split_full;    // vocab chunks per full wave
+    int32_t full_waves;
+    int32_t rem_m;         // row tiles of the last wave (0: none)
+    int32_t split_rem;     // vocab chunks of the last wave
+    int32_t waves;         // full_waves + (rem_m > 0)
+};
+
+// Host-side planner (pure arithmetic, no CUDA calls).
+ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms);
+size_t plan_workspace_bytes(const ScorePlan& p);
+
+// Work unit of CTA `cta` in wave `wave`: returns false when the CTA idles in that wave.
+__host__ __device__ inline bool plan_unit(const ScorePlan& p, int wave, int cta,
+                                          int* row_tile, int* n_begin, int* n_end) {
+    int gm, s, base;
+    if (wave < p.full_waves) { gm = p.group_m; s = p.split_full; base = wave * p.group_m; }
+    else                     { gm = p.rem_m;   s = p.split_rem;  base = p.full_waves * p.group_m; }
+    if (gm <= 0 || cta >= gm * s) return false;
+    const int i = cta % gm, c = cta / gm;
+    *row_tile = base + i;
+    *n_begin = (int)(((int64_t)c * p.vocab_tiles) / s);
+    *n_end   = (int)(((int64_t)(c + 1) * p.vocab_tiles) / s);
+    return true;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TimedLaunch { cudaEvent_t start, stop; };
+
+}  // namespace specs
+
+struct specs_ctx {
+    int device = 0;
+    int num_sms = 0;
+    int engine = SPECS_ENGINE_TCGEN05;
+    uint32_t* d_status = nullptr;          // device status word (SPECS_DEV_* bits)
+    specs::EncodeTiledFn encode_tiled = nullptr;
+    // grow-only device arena for specs_beam_step_host
+    void* arena = nullptr;
+    size_t arena_bytes = 0;
+    // optional per-launch timing of the tensor-core kernel
+    bool timing = false;
+    std::vector<specs::TimedLaunch> timed;
+    size_t timed_used = 0;
+};
+
+namespace specs {
+
+// ---- kernel launchers (each enqueues on `stream`, returns a specs_status) ---------------------
+int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan, const void* hidden, const void* w_vocab,
+                         const int32_t* token_ids, float* workspace, cudaStream_t stream);
+int launch_score_simt(specs_ctx* ctx, const void* hidden, const void* w_vocab, const int32_t* token_ids,
+                      int64_t rows, int32_t d, int32_t V, float* tok_logprob, cudaStream_t stream);
+int launch_merge(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, const int32_t* token_ids,
+                 float* tok_logprob, cudaStream_t stream);
+int launch_block_sums(const float* per_token, const int64_t* block_offsets, int32_t B,
+                      float* out, double* out_f64, cudaStream_t stream);
+int launch_subsample(const void* lp_target, const void* lp_gen, bool lp_is_f64, const float* reward,
+                     const int32_t* cand_offsets, int32_t P, float beta, const float* uniforms,
+                     int32_t* chosen, float* weights, float tau, uint8_t* accept, cudaStream_t stream);
+int launch_accept(const float* reward, const int32_t* cand_offsets, int32_t P, float tau,
+                  uint8_t* accept, cudaStream_t stream);
+
+inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? SPECS_OK : SPECS_ERR_CUDA; }
+
+}  // namespace specs

@@ -1,0 +1,309 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Run with -m gpu on a B200."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import specs_oracle as O
+from paper_2506_15733_b200 import binding
+from paper_2506_15733_b200 import inputs as I
+from tests.gpu_util import BLK_RTOL, MARGIN, TOK_ATOL, DeviceStep, assert_step_matches
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(0)
+    yield c
+    assert c.device_status() == 0, "device status word not clean at the end of the module"
+    c.close()
+
+
+def oracle_step(x, beta, tau, with_draft=True):
+    return O.beam_step(x.hidden, x.w_vocab, x.token_ids, x.block_offsets, x.cand_offsets,
+                       x.draft_tok_logprob if with_draft else None, x.reward, beta, x.uniforms, tau)
+
+
+def small_config(name, rows_per_block, problems, beams, d, V, seed, **kw):
+    return I.StepConfig(name, seed, problems, beams, rows_per_block, d, V, kw.pop("w_sigma", 0.05), **kw)
+
+
+# ------------------------------------------------------------------------------- tiny, both engines
+
+@pytest.mark.parametrize("engine", [binding.ENGINE_SIMT, binding.ENGINE_TCGEN05])
+def test_tiny_config_full_step(ctx, engine):
+    x = I.make_step_inputs(I.CONFIGS["tiny"])
+    ctx.set_engine(engine)
+    try:
+        got = DeviceStep(ctx, x).step(1.0, 0.7)
+    finally:
+        ctx.set_engine(binding.ENGINE_TCGEN05)
+    want = oracle_step(x, 1.0, 0.7)
+    info = assert_step_matches(got, want, x.cand_offsets, x.block_offsets)
+    w_err = np.abs(got["weights"] - want["weights"]).max()
+    assert w_err < 5e-3, w_err
+    assert abs(got["weights"].sum() - 1.0) < 1e-5
+    assert ctx.device_status() == 0
+
+
+# ------------------------------------------------------------------------------- tile edges and ragged tails
+
+EDGE_CASES = [
+    # rows/block range, problems, beams, d, V
+    ((1, 1), 1, 1, 8, 8),            # a single row, a single k-block with a 56-element tail, 8 vocab entries
+    ((127, 127), 1, 1, 72, 1000),    # one row short of a tile; d and V with ragged tails
+    ((129, 129), 1, 1, 64, 1032),    # one row over a tile; V = 4 tiles + 8
+    ((3, 40), 3, 5, 256, 2500),      # ragged blocks, several tiles, vocab tail of 196
+    ((16, 16), 2, 4, 520, 257),      # vocab tile with a single valid column in its last tile
+    ((50, 50), 1, 6, 1024, 4096),    # exact multiples everywhere
+]
+
+
+@pytest.mark.parametrize("blk,P,n,d,V", EDGE_CASES)
+def test_edge_shapes(ctx, blk, P, n, d, V):
+    cfg = small_config("edge", blk, P, n, d, V, seed=4000 + d + V)
+    x = I.make_step_inputs(cfg)
+    got = DeviceStep(ctx, x).step(1.0, 0.5)
+    want = oracle_step(x, 1.0, 0.5)
+    assert_step_matches(got, want, x.cand_offsets, x.block_offsets)
+    assert ctx.device_status() == 0
+
+
+def test_empty_blocks_and_empty_problem(ctx):
+    cfg = small_config("holes", (5, 9), 3, 3, 64, 300, seed=4100)
+    x = I.make_step_inputs(cfg)
+    # make block 2 and block 7 empty, and problem 1 empty (its three blocks move to problem 2)
+    lens = np.diff(x.block_offsets)
+    lens[2] = 0
+    lens[7] = 0
+    x.block_offsets = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    rows = int(x.block_offsets[-1])
+    x.hidden, x.token_ids, x.draft_tok_logprob = x.hidden[:rows], x.token_ids[:rows], x.draft_tok_logprob[:rows]
+    x.cand_offsets = np.array([0, 3, 3, 9], dtype=np.int32)
+    got = DeviceStep(ctx, x).step(2.0, 0.4)
+    want = oracle_step(x, 2.0, 0.4)
+    assert_step_matches(got, want, x.cand_offsets, x.block_offsets)
+    assert got["blk_logprob"][2] == 0.0 and got["blk_logprob"][7] == 0.0
+    assert got["chosen"][1] == -1 and got["accept"][1] == 0
+
+
+def test_zero_rows_is_a_noop(ctx):
+    dev = "cuda:0"
+    w = binding.bf16_bits_to_device(np.zeros((16, 8), np.uint16), dev)
+    h = torch.empty((0, 8), dtype=torch.bfloat16, device=dev)
+    ids = torch.empty((0,), dtype=torch.int32, device=dev)
+    offs = torch.zeros(3, dtype=torch.int64, device=dev)
+    tok = torch.empty((0,), dtype=torch.float32, device=dev)
+    blk = torch.full((2,), 5.0, dtype=torch.float32, device=dev)
+    ctx.specs_score_blocks(h, w, ids, offs, tok, blk, None, None)
+    torch.cuda.synchronize()
+    assert blk.tolist() == [0.0, 0.0]
+
+
+# ------------------------------------------------------------------------------- several waves of work units
+
+@pytest.mark.parametrize("rows_total,d,V", [(20000, 64, 1000), (10000, 1536, 2048), (40000, 128, 520)])
+def test_multi_wave_plans(ctx, rows_total, d, V):
+    sms = ctx.sm_count()
+    plan = binding.score_plan(rows_total, d, V, sms)
+    assert plan["waves"] >= 2, plan
+    blocks = 40
+    cfg = small_config("waves", (rows_total // blocks, rows_total // blocks), 4, blocks // 4, d, V,
+                       seed=4200 + d, w_sigma=0.5 / math.sqrt(d) * 4)
+    x = I.make_step_inputs(cfg)
+    got = DeviceStep(ctx, x).step(1.0, 0.6)
+    want = oracle_step(x, 1.0, 0.6)
+    assert_step_matches(got, want, x.cand_offsets, x.block_offsets)
+    assert ctx.device_status() == 0
+
+
+# ------------------------------------------------------------------------------- device-detected conditions
+
+def test_out_of_range_token_is_nan_and_flagged(ctx):
+    cfg = small_config("badid", (8, 8), 1, 2, 64, 300, seed=4300)
+    x = I.make_step_inputs(cfg)
+    x.token_ids = x.token_ids.copy()
+    x.token_ids[3] = 300
+    x.token_ids[9] = -2
+    for engine in (binding.ENGINE_TCGEN05, binding.ENGINE_SIMT):
+        ctx.set_engine(engine)
+        try:
+            s = DeviceStep(ctx, x)
+            s.score()
+            torch.cuda.synchronize()
+        finally:
+            ctx.set_engine(binding.ENGINE_TCGEN05)
+        lp = s.tok_lp.cpu().numpy()
+        assert np.isnan(lp[3]) and np.isnan(lp[9])
+        ok = np.ones(16, bool)
+        ok[[3, 9]] = False
+        want = O.token_logprobs(x.hidden, x.w_vocab, x.token_ids)
+        assert np.abs(lp[ok] - want[ok]).max() <= TOK_ATOL
+        assert ctx.device_status() == binding.DEV_TOKEN_RANGE
+        assert ctx.device_status() == 0                       # reading clears it
+
+
+def test_host_side_argument_errors(ctx):
+    cfg = small_config("args", (4, 4), 1, 2, 64, 300, seed=4400)
+    x = I.make_step_inputs(cfg)
+    s = DeviceStep(ctx, x)
+    with pytest.raises(binding.SpecsError) as e:
+        ctx.specs_score_blocks(s.hidden, s.w_vocab, s.token_ids, s.block_offsets, s.tok_lp, s.blk_lp, None,
+                               s.workspace[:64])
+    assert e.value.status == 4                                # workspace too small
+    with pytest.raises(binding.SpecsError) as e:
+        ctx.specs_score_blocks(s.hidden, s.w_vocab, None, s.block_offsets, s.tok_lp, s.blk_lp, None, s.workspace)
+    assert e.value.status == 1
+    odd = s.hidden.view(torch.int16).reshape(-1)[4:4 + 7 * 64].view(torch.bfloat16).reshape(7, 64)   # 8-byte aligned
+    with pytest.raises(binding.SpecsError) as e:
+        ctx.specs_score_blocks(odd, s.w_vocab, s.token_ids, s.block_offsets, s.tok_lp, None, None, s.workspace)
+    assert e.value.status == 3
+    bad_d = torch.zeros((8, 12), dtype=torch.bfloat16, device="cuda:0")
+    with pytest.raises(binding.SpecsError) as e:
+        ctx.specs_score_blocks(bad_d, bad_d, s.token_ids, s.block_offsets, s.tok_lp, None, None, s.workspace)
+    assert e.value.status == 2
+    torch.cuda.synchronize()
+    assert torch.isnan(s.tok_lp).all()                        # nothing was launched, outputs untouched
+
+
+# ------------------------------------------------------------------------------- selection kernels alone
+
+@pytest.mark.parametrize("beta", [0.0, 1.0, 4.0, 1.0e4])
+@pytest.mark.parametrize("f64", [False, True])
+def test_subsample_matches_oracle_on_many_problems(ctx, beta, f64):
+    rng = np.random.Generator(np.random.Philox(key=[4500, int(beta) + 7 * f64]))
+    sizes = rng.integers(0, 70, size=3000)                    # includes empty problems and n > 32
+    cand = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    B = int(cand[-1])
+    lp_t = rng.uniform(-4000, -5, B)
+    lp_g = lp_t + rng.normal(0, 3.0, B)
+    if not f64:
+        lp_t, lp_g = lp_t.astype(np.float32), lp_g.astype(np.float32)
+    r = rng.random(B).astype(np.float32)
+    u = I.draw_uniforms(4501, B)
+    dev = "cuda:0"
+    t = lambda a: torch.from_numpy(a).to(dev)
+    chosen = torch.empty(len(sizes), dtype=torch.int32, device=dev)
+    wts = torch.empty(B, dtype=torch.float32, device=dev)
+    acc = torch.empty(len(sizes), dtype=torch.uint8, device=dev)
+    ctx.specs_subsample(t(lp_t), t(lp_g), t(r), t(cand), beta, t(u), chosen, wts, 0.97, acc)
+    torch.cuda.synchronize()
+    S = O.scores(lp_t, lp_g, r, beta)
+    want_c, margin = O.gumbel_pick(S, u, cand)
+    want_w = O.weights(S, cand)
+    got_c = chosen.cpu().numpy()
+    sure = margin > MARGIN
+    assert sure.sum() > 2000
+    assert np.array_equal(got_c[sure], want_c[sure])
+    assert np.array_equal(got_c[sizes == 0], np.full((sizes == 0).sum(), -1))
+    assert np.all((got_c[sizes > 0] >= 0) & (got_c[sizes > 0] < sizes[sizes > 0]))
+    assert np.abs(wts.cpu().numpy() - want_w).max() < 1e-6
+    assert np.array_equal(acc.cpu().numpy(), O.accept_flags(r, cand, 0.97))
+
+
+def test_subsample_same_generator_and_null_outputs(ctx):
+    # pi_gen = pi_target: scores collapse to beta * r (text after Eq. 1); weights and accept are optional
+    rng = np.random.Generator(np.random.Philox(key=[4600, 1]))
+    n, P = 16, 500
+    cand = (np.arange(P + 1) * n).astype(np.int32)
+    r = rng.beta(2, 2, n * P).astype(np.float32)
+    u = I.draw_uniforms(4601, n * P)
+    dev = "cuda:0"
+    t = lambda a: torch.from_numpy(a).to(dev)
+    chosen = torch.empty(P, dtype=torch.int32, device=dev)
+    wts = torch.empty(n * P, dtype=torch.float32, device=dev)
+    ctx.specs_subsample(None, None, t(r), t(cand), 4.0, t(u), chosen, wts)
+    chosen2 = torch.empty(P, dtype=torch.int32, device=dev)
+    ctx.specs_subsample(None, None, t(r), t(cand), 4.0, t(u), chosen2, None)
+    torch.cuda.synchronize()
+    S = O.scores(None, None, r, 4.0)
+    want_c, margin = O.gumbel_pick(S, u, cand)
+    sure = margin > MARGIN
+    assert np.array_equal(chosen.cpu().numpy()[sure], want_c[sure])
+    assert np.array_equal(chosen.cpu().numpy(), chosen2.cpu().numpy())
+    e = np.exp(4.0 * r.astype(np.float64)).reshape(P, n)
+    assert np.abs(wts.cpu().numpy().reshape(P, n) - e / e.sum(1, keepdims=True)).max() < 1e-6
+
+
+@pytest.mark.parametrize("beta", [0.0, 1.0, 4.0])
+def test_gpu_sampler_chi_squared(ctx, beta):
+    # empirical pick frequencies of the CUDA sampler against the closed-form weights
+    from scipy import stats
+    LP = np.array([-20.0, -21.0, -19.5, -22.0, -20.5, -23.0, -19.0, -21.5], dtype=np.float32)
+    LQ = np.array([-20.5, -20.0, -20.0, -21.0, -21.5, -22.0, -20.0, -21.0], dtype=np.float32)
+    r = np.array([0.1, 0.6, 0.3, 0.9, 0.5, 0.7, 0.2, 0.4], dtype=np.float32)
+    n, draws = 8, 400_000
+    cand = (np.arange(draws + 1) * n).astype(np.int32)
+    u = I.draw_uniforms(4700 + int(beta), n * draws)
+    dev = "cuda:0"
+    t = lambda a: torch.from_numpy(a).to(dev)
+    chosen = torch.empty(draws, dtype=torch.int32, device=dev)
+    ctx.specs_subsample(t(np.tile(LP, draws)), t(np.tile(LQ, draws)), t(np.tile(r, draws)), t(cand), beta, t(u),
+                        chosen, None)
+    torch.cuda.synchronize()
+    counts = np.bincount(chosen.cpu().numpy(), minlength=n)
+    expected = draws * O.weights(O.scores(LP, LQ, r, beta), np.array([0, n]))
+    assert expected.min() >= 5
+    assert stats.chisquare(counts, expected).pvalue > 1e-3, (counts, expected)
+
+
+def test_accept_threshold_sweep(ctx):
+    x = I.make_step_inputs(I.CONFIGS["batched"], with_weights=False)
+    dev = "cuda:0"
+    r = torch.from_numpy(x.reward).to(dev)
+    cand = torch.from_numpy(x.cand_offsets).to(dev)
+    acc = torch.empty(32, dtype=torch.uint8, device=dev)
+    prev = None
+    for tau in (-1.0,) + I.CONFIGS["batched"].taus + (1.0,):
+        ctx.specs_accept(r, cand, tau, acc)
+        torch.cuda.synchronize()
+        got = acc.cpu().numpy()
+        assert np.array_equal(got, O.accept_flags(x.reward, x.cand_offsets, tau))
+        if prev is not None:
+            assert np.all(got <= prev)
+        prev = got
+    assert prev.sum() == 0                                    # tau = 1: never switches to the draft
+
+
+def test_block_sums_kernel(ctx):
+    rng = np.random.Generator(np.random.Philox(key=[4800, 1]))
+    lens = rng.integers(0, 600, 300)
+    offs = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    v = rng.uniform(-12, 0, int(offs[-1])).astype(np.float32)
+    dev = "cuda:0"
+    o32 = torch.empty(300, dtype=torch.float32, device=dev)
+    o64 = torch.empty(300, dtype=torch.float64, device=dev)
+    ctx.specs_block_sums(torch.from_numpy(v).to(dev), torch.from_numpy(offs).to(dev), o32, o64)
+    torch.cuda.synchronize()
+    want = O.block_sums(v, offs)
+    assert np.abs(o64.cpu().numpy() - want).max() < 1e-9
+    assert np.array_equal(o32.cpu().numpy(), want.astype(np.float32)) or \
+        np.abs(o32.cpu().numpy() - want).max() <= 1e-6 * np.abs(want).max()
+
+
+# ------------------------------------------------------------------------------- host-buffer entry point
+
+def test_beam_step_host_equals_device_calls(ctx):
+    cfg = small_config("host", (3, 40), 3, 5, 256, 2500, seed=4900)
+    x = I.make_step_inputs(cfg)
+    want_dev = DeviceStep(ctx, x).step(1.5, 0.55)
+    rows, B, P = x.rows, x.blocks, 3
+    tok = np.empty(rows, np.float32); blk = np.empty(B, np.float64); wts = np.empty(B, np.float32)
+    cho = np.empty(P, np.int32); acc = np.empty(P, np.uint8)
+    w_dev = binding.bf16_bits_to_device(x.w_vocab, "cuda:0")
+    for _ in range(2):                                        # the second call reuses the arena
+        ctx.specs_beam_step_host(x.hidden, w_dev, x.token_ids, x.block_offsets, x.cand_offsets,
+                                 x.draft_tok_logprob, x.reward, x.uniforms, 1.5, 0.55, tok, blk, wts, cho, acc)
+        assert np.array_equal(tok, want_dev["tok_logprob"])
+        assert np.array_equal(blk, want_dev["blk_logprob_f64"])
+        assert np.array_equal(wts, want_dev["weights"])
+        assert np.array_equal(cho, want_dev["chosen"]) and np.array_equal(acc, want_dev["accept"])
+    bad = x.block_offsets.copy()
+    bad[2] = bad[3] + 1
+    with pytest.raises(binding.SpecsError) as e:
+        ctx.specs_beam_step_host(x.hidden, w_dev, x.token_ids, bad, x.cand_offsets, x.draft_tok_logprob, x.reward,
+                                 x.uniforms, 1.5, 0.55, tok, blk, wts, cho, acc)
+    assert e.value.status == 5

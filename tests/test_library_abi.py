@@ -1,0 +1,97 @@
+"""CPU checks of the shared library: it builds, loads, exports every symbol the header
+declares, and its host-side work-unit planner tiles the problem exactly once."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2506_15733_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load_library()
+
+
+def header_functions():
+    text = open(os.path.join(ROOT, "include", "specs.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(specs_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported_and_bound(lib):
+    names = header_functions()
+    assert len(names) >= 15
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in specs.h but not exported"
+    assert sorted(binding.SIGNATURES) == names, "binding.SIGNATURES and specs.h disagree"
+
+
+def test_status_strings(lib):
+    assert binding.status_string(0) == "ok"
+    seen = {binding.status_string(i) for i in range(0, 11)}
+    assert len(seen) == 11 and "unknown status" not in seen
+    assert binding.status_string(99) == "unknown status"
+
+
+def test_host_validation_without_a_device(lib):
+    out = (ctypes.c_int32 * 12)()
+    assert lib.specs_score_plan(128, 12, 100, 148, out) == 2        # d % 8 != 0
+    assert lib.specs_score_plan(-1, 16, 100, 148, out) == 2
+    assert lib.specs_score_plan(128, 16, 0, 148, out) == 2
+    assert lib.specs_score_plan(128, 16, 100, 148, None) == 1
+    # calls that need a context refuse a NULL one instead of crashing
+    assert lib.specs_destroy(None) == 0
+    assert lib.specs_set_engine(None, 0) == 1
+    assert lib.specs_score_workspace_bytes(None, 128, 16, 100) == 0
+    assert lib.specs_accept(None, None, None, 1, 0.5, None, None) == 1
+
+
+PLAN_CASES = [
+    (64, 256, 1024, 148), (1024, 3584, 151936, 148), (20893, 3584, 151936, 148),
+    (65536, 1536, 151936, 148), (65536, 3584, 151936, 148), (131072, 5120, 152064, 148),
+    (1, 8, 8, 148), (129, 72, 1000, 148), (20000, 64, 1000, 148), (10000, 1536, 2048, 148),
+    (777, 128, 300, 7), (5000, 4096, 70000, 132), (128 * 148 + 1, 64, 257, 148),
+]
+
+
+@pytest.mark.parametrize("rows,d,V,sms", PLAN_CASES)
+def test_plan_covers_every_tile_exactly_once(lib, rows, d, V, sms):
+    p = binding.score_plan(rows, d, V, sms)
+    assert p["row_tiles"] == -(-rows // 128) and p["vocab_tiles"] == -(-V // 256) and p["k_blocks"] == -(-d // 64)
+    assert p["grid"] == sms and p["waves"] == p["full_waves"] + (1 if p["rem_m"] else 0)
+    assert p["group_m"] * p["split_full"] <= sms
+    assert p["full_waves"] * p["group_m"] + p["rem_m"] == p["row_tiles"]
+    if p["rem_m"]:
+        assert 1 <= p["split_rem"] and p["rem_m"] * p["split_rem"] <= sms
+    assert p["workspace_bytes"] == p["waves"] * sms * 3 * 128 * 4
+    assert p["workspace_bytes"] < 64 * rows + (1 << 20)              # never anything like rows x V
+    covered = {}
+    busiest = 0
+    for w in range(p["waves"]):
+        for c in range(sms):
+            mt, nb, ne = binding.score_plan_unit(rows, d, V, sms, w, c)
+            if mt < 0:
+                continue
+            assert 0 <= mt < p["row_tiles"] and 0 <= nb < ne <= p["vocab_tiles"]
+            for n in range(nb, ne):
+                assert (mt, n) not in covered
+                covered[(mt, n)] = (w, c)
+            busiest = max(busiest, ne - nb)
+    assert len(covered) == p["row_tiles"] * p["vocab_tiles"]
+
+
+def test_plan_balance_on_the_benchmark_shapes(lib):
+    # makespan in tiles per CTA versus the ideal total / grid
+    for rows, d, V in [(1024, 3584, 151936), (65536, 3584, 151936), (131072, 5120, 152064), (65536, 1536, 151936)]:
+        p = binding.score_plan(rows, d, V, 148)
+        span = 0
+        for w in range(p["waves"]):
+            span += max(ne - nb for mt, nb, ne in
+                        (binding.score_plan_unit(rows, d, V, 148, w, c) for c in range(148)) if mt >= 0)
+        ideal = p["row_tiles"] * p["vocab_tiles"] / 148
+        assert span <= 1.06 * ideal + 1, (rows, d, V, span, ideal, p)
