@@ -377,12 +377,14 @@ int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan, const void* hidd
     st = encode_bf16_2d(ctx, &map_w, w_vocab, (uint64_t)plan.d, (uint64_t)plan.V, kBlockK, kBlockN);
     if (st != SPECS_OK) return st;
 
-    static bool attr_set = false;
-    if (!attr_set) {
+    // The opt-in to more than 48 KB of dynamic shared memory is a per-device function attribute.
+    static bool attr_set[64] = {};
+    const int dev_slot = ctx->device & 63;
+    if (!attr_set[dev_slot]) {
         cudaError_t e = cudaFuncSetAttribute(score_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kSmemBytes);
         if (e != cudaSuccess) return SPECS_ERR_CUDA;
-        attr_set = true;
+        attr_set[dev_slot] = true;
     }
     TimedLaunch* tl = nullptr;
     if (ctx->timing) {
