@@ -198,6 +198,43 @@ int specs_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_
 int specs_score_plan_unit(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t wave, int32_t cta,
                           int32_t* h_out3);
 
+/* Block scoring for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this entry point exists for deployment, not for the method.)
+ *
+ * Who needs it: a serving process that handed the whole GPU to its own memory pool
+ * at start-up (nothing is left for cudaMalloc to return), or a step loop that must
+ * never meet the device-wide synchronisation cudaMalloc / cudaFree imply.  Such a
+ * caller can neither create a specs_ctx (creation allocates the status word) nor
+ * supply a workspace, so this call takes neither: the scratch of the scoring kernel
+ * is a fixed array of SPECS_NOALLOC_SCRATCH_BYTES inside the library's device image,
+ * which every GPU that loads the library holds until the process exits.  The call
+ * itself, and everything it runs, calls no cudaMalloc, cudaFree or other allocating
+ * routine; inputs and outputs are the caller's buffers as in specs_score_blocks
+ * (same meaning, layout and requirements), always on the tensor-core engine, on the
+ * CURRENT device.
+ *
+ *   status_word  device uint32 that receives SPECS_DEV_* bits by atomic OR (never
+ *                cleared by the library); NULL sends them to an internal word that
+ *                cannot be read back.
+ *
+ * Limits and sharing:
+ *   - the plan for (rows, d, V) must fit the fixed scratch (waves x SMs x 1536 bytes
+ *     <= SPECS_NOALLOC_SCRATCH_BYTES; about 110 000 rows at d = 3584 and 85 000 at
+ *     d = 5120 on a 148-SM part); larger problems return SPECS_ERR_LIMIT and launch
+ *     nothing.  Split the rows over several calls instead.
+ *   - all calls on a device share the one array, which still holds the previous
+ *     call's contents.  Nothing in it has to start at zero (each slot is written
+ *     before it is read within a call), but calls whose kernels overlap on the GPU,
+ *     e.g. on different streams, race on it: serialise them.
+ *   - the first call on each device resolves the array's device address
+ *     (cudaGetSymbolAddress) and the driver entry point it needs; make that first
+ *     call before starting any stream capture. */
+#define SPECS_NOALLOC_SCRATCH_BYTES (4u << 20)
+int specs_score_blocks_noalloc(const void* hidden, const void* W_vocab, const int32_t* token_ids,
+                               const int64_t* block_offsets, int64_t rows, int32_t d, int32_t V, int32_t B,
+                               float* tok_logprob, float* blk_logprob, double* blk_logprob_f64,
+                               uint32_t* status_word, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

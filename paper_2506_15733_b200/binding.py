@@ -44,6 +44,7 @@ SIGNATURES = {
                                        _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "specs_set_timing": (C.c_int, [_vp, C.c_int]),
     "specs_score_kernel_ms": (C.c_float, [_vp, C.POINTER(_i32)]),
+    "specs_score_blocks_noalloc": (C.c_int, [_vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]),
     "specs_score_plan": (C.c_int, [_i64, _i32, _i32, _i32, C.POINTER(_i32)]),
     "specs_score_plan_unit": (C.c_int, [_i64, _i32, _i32, _i32, _i32, _i32, C.POINTER(_i32)]),
 }
@@ -204,6 +205,25 @@ class Context:
             _ptr(h_gen_tok_logprob), _ptr(h_reward), _ptr(h_uniforms), rows, d, V, B, P, float(beta), float(tau),
             _ptr(h_tok_logprob), _ptr(h_blk_logprob), _ptr(h_weights), _ptr(h_chosen), _ptr(h_accept), _stream()),
             "specs_beam_step_host")
+
+
+NOALLOC_SCRATCH_BYTES = 4 << 20
+
+
+def specs_score_blocks_noalloc(hidden, w_vocab, token_ids, block_offsets, tok_logprob,
+                               blk_logprob=None, blk_logprob_f64=None, status_word=None):
+    """Context-free, allocation-free scoring on the current CUDA device (see specs.h).
+
+    For hosts that cannot call cudaMalloc: the kernel's scratch is a fixed array inside the
+    library, shared by all calls on the device, so calls must not overlap on the GPU and
+    problems beyond the fixed size raise SpecsError(SPECS_ERR_LIMIT).
+    """
+    rows, d = hidden.shape
+    V = w_vocab.shape[0]
+    B = block_offsets.shape[0] - 1
+    _check(load_library().specs_score_blocks_noalloc(
+        _ptr(hidden), _ptr(w_vocab), _ptr(token_ids), _ptr(block_offsets), rows, d, V, B, _ptr(tok_logprob),
+        _ptr(blk_logprob), _ptr(blk_logprob_f64), _ptr(status_word), _stream()), "specs_score_blocks_noalloc")
 
 
 # ---------------------------------------------------------------------------- torch helpers (marshalling only)
