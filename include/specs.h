@@ -70,6 +70,14 @@ int specs_destroy(specs_ctx* ctx);
 /* Select the scoring engine for later specs_score_blocks calls on this context. */
 int specs_set_engine(specs_ctx* ctx, int engine);
 
+/* Length, in elements of d, of one tensor-core accumulation chunk (a multiple of
+ * 64; default 512; 0 = accumulate the whole of d in one go).  The tensor core adds
+ * into its fp32 accumulator with truncation, which biases long reductions of large
+ * logits (about -5e-3 at |logit| = 700, d = 5120); the kernel therefore restarts the
+ * accumulator every chunk and sums the chunks in registers with round-to-nearest,
+ * which divides the bias by the number of chunks.  Shorter chunks cost epilogue time. */
+int specs_set_accum_chunk(specs_ctx* ctx, int32_t k_elements);
+
 /* Number of SMs the context schedules over (also the persistent grid size). */
 int specs_sm_count(const specs_ctx* ctx);
 
@@ -218,7 +226,7 @@ int specs_score_plan_unit(int64_t rows, int32_t d, int32_t V, int32_t num_sms, i
  *                cannot be read back.
  *
  * Limits and sharing:
- *   - the plan for (rows, d, V) must fit the fixed scratch (waves x SMs x 1536 bytes
+ *   - the plan for (rows, d, V) must fit the fixed scratch (waves x SMs x 3072 bytes
  *     <= SPECS_NOALLOC_SCRATCH_BYTES; about 110 000 rows at d = 3584 and 85 000 at
  *     d = 5120 on a 148-SM part); larger problems return SPECS_ERR_LIMIT and launch
  *     nothing.  Split the rows over several calls instead.
@@ -229,7 +237,7 @@ int specs_score_plan_unit(int64_t rows, int32_t d, int32_t V, int32_t num_sms, i
  *   - the first call on each device resolves the array's device address
  *     (cudaGetSymbolAddress) and the driver entry point it needs; make that first
  *     call before starting any stream capture. */
-#define SPECS_NOALLOC_SCRATCH_BYTES (4u << 20)
+#define SPECS_NOALLOC_SCRATCH_BYTES (8u << 20)
 int specs_score_blocks_noalloc(const void* hidden, const void* W_vocab, const int32_t* token_ids,
                                const int64_t* block_offsets, int64_t rows, int32_t d, int32_t V, int32_t B,
                                float* tok_logprob, float* blk_logprob, double* blk_logprob_f64,

@@ -31,6 +31,7 @@ SIGNATURES = {
     "specs_create": (C.c_int, [C.POINTER(_vp), C.c_int]),
     "specs_destroy": (C.c_int, [_vp]),
     "specs_set_engine": (C.c_int, [_vp, C.c_int]),
+    "specs_set_accum_chunk": (C.c_int, [_vp, _i32]),
     "specs_sm_count": (C.c_int, [_vp]),
     "specs_score_workspace_bytes": (C.c_size_t, [_vp, _i64, _i32, _i32]),
     "specs_score_blocks": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp,
@@ -137,6 +138,9 @@ class Context:
     def set_engine(self, engine: int):
         _check(self._lib.specs_set_engine(self._h, int(engine)), "specs_set_engine")
 
+    def set_accum_chunk(self, k_elements: int):
+        _check(self._lib.specs_set_accum_chunk(self._h, int(k_elements)), "specs_set_accum_chunk")
+
     def sm_count(self) -> int:
         return int(self._lib.specs_sm_count(self._h))
 
@@ -207,7 +211,7 @@ class Context:
             "specs_beam_step_host")
 
 
-NOALLOC_SCRATCH_BYTES = 4 << 20
+NOALLOC_SCRATCH_BYTES = 8 << 20
 
 
 def specs_score_blocks_noalloc(hidden, w_vocab, token_ids, block_offsets, tok_logprob,

@@ -9,7 +9,7 @@
 namespace specs {
 
 // ---------------------------------------------------------------------------------- planner
-ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms) {
+ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t chunk_kblocks) {
     ScorePlan p;
     std::memset(&p, 0, sizeof(p));
     p.rows = rows; p.d = d; p.V = V;
@@ -17,6 +17,7 @@ ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms) {
     p.vocab_tiles = (V + kBlockN - 1) / kBlockN;
     p.k_blocks = (d + kBlockK - 1) / kBlockK;
     p.grid = num_sms;
+    p.chunk_kblocks = (chunk_kblocks > 0 && chunk_kblocks < p.k_blocks) ? chunk_kblocks : p.k_blocks;
     if (p.row_tiles == 0) return p;
 
     // Full waves: the fewest vocabulary chunks s (hence the most row tiles gm = grid / s sharing
@@ -165,6 +166,13 @@ int specs_set_engine(specs_ctx* ctx, int engine) {
     return SPECS_OK;
 }
 
+int specs_set_accum_chunk(specs_ctx* ctx, int32_t k_elements) {
+    if (!ctx) return SPECS_ERR_NULL;
+    if (k_elements < 0 || (k_elements % kBlockK) != 0) return SPECS_ERR_SHAPE;
+    ctx->chunk_kblocks = k_elements / kBlockK;               // 0: one accumulator over the whole of d
+    return SPECS_OK;
+}
+
 int specs_sm_count(const specs_ctx* ctx) { return ctx ? ctx->num_sms : 0; }
 
 size_t specs_score_workspace_bytes(const specs_ctx* ctx, int64_t rows, int32_t d, int32_t V) {
@@ -216,7 +224,7 @@ int specs_score_blocks(specs_ctx* ctx, const void* hidden, const void* W_vocab, 
             st = launch_score_simt(ctx, hidden, W_vocab, token_ids, rows, d, V, tok_logprob, stream);
             if (st != SPECS_OK) return st;
         } else {
-            const ScorePlan plan = make_score_plan(rows, d, V, ctx->num_sms);
+            const ScorePlan plan = make_score_plan(rows, d, V, ctx->num_sms, ctx->chunk_kblocks);
             if (!workspace) return SPECS_ERR_NULL;
             if (workspace_bytes < plan_workspace_bytes(plan)) return SPECS_ERR_WORKSPACE;
             st = launch_score_tcgen05(ctx, plan, hidden, W_vocab, token_ids, static_cast<float*>(workspace), stream);

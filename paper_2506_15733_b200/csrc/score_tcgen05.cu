@@ -6,15 +6,25 @@
 // This is the "computing logits of each token" step of scoring a drafted block with the
 // target model (Section 2 of the paper; Appendix E.3 restricts it to the new block's tokens).
 //
-// One persistent CTA per SM, 192 threads, three roles:
+// One persistent CTA per SM, 384 threads (three warpgroups), three roles:
 //   warp 0      TMA producer: cp.async.bulk.tensor loads of a 128x64 hidden tile and a 256x64
 //               W tile per k-block into a 4-stage, 128-byte-swizzled shared-memory ring.
-//   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32);
-//               the accumulator is one of two 128-lane x 256-column TMEM buffers, so the
-//               epilogue of vocabulary tile j overlaps the MMAs of tile j+1.
-//   warps 2-5   epilogue: thread = one row (TMEM lane).  tcgen05.ld 32 columns at a time,
-//               running max / rescaled sum of 2^x / select of the drafted id's logit, all in
-//               registers across the CTA's run of vocabulary tiles.
+//   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32)
+//               into one of two 128-lane x 256-column TMEM buffers.  The reduction over d is
+//               cut into chunks of plan.chunk_kblocks k-blocks; every chunk starts a fresh
+//               accumulator and alternates between the two buffers.
+//   warps 4-11  epilogue: thread = one row (TMEM lane) x one half (128 columns) of the tile.
+//               After each chunk it adds the chunk's partial logits into fp32 registers
+//               (round-to-nearest), which releases the TMEM buffer for the chunk after next;
+//               after the last chunk it runs, on those registers, the online update of
+//               running max / rescaled sum of 2^x / select of the drafted id's logit.  The
+//               state stays in registers across the CTA's run of vocabulary tiles.
+//
+// Why chunks: the tensor core adds each K=16 group of products into its fp32 accumulator with
+// truncation, so a long reduction carries a bias proportional to the accumulator's magnitude
+// times the number of accumulations (about -5e-3 on logits near 700 at d = 5120).  Restarting
+// the accumulator every 512 elements and summing the chunks in registers with round-to-nearest
+// divides that bias by the number of chunks.
 // Every mbarrier wait is bounded; on expiry the CTA raises SPECS_DEV_TIMEOUT, all roles leave
 // their loops, the producer waits (bounded) for its copies in flight, TMEM is freed and the
 // kernel returns.
@@ -30,8 +40,9 @@ constexpr int kUmmaK = 16;
 constexpr uint32_t kABytes = kBlockM * kBlockK * 2;      // 16 KB
 constexpr uint32_t kBBytes = kBlockN * kBlockK * 2;      // 32 KB
 constexpr uint32_t kStageBytes = kABytes + kBBytes;      // 48 KB
-constexpr int kThreads = 192;
-constexpr int kEpilogueThreads = 128;
+constexpr int kThreads = 384;                            // three warpgroups: control, epilogue, epilogue
+constexpr int kEpilogueThreads = 256;
+constexpr int kHalfN = kBlockN / 2;                      // columns per epilogue thread
 constexpr uint32_t kTmemCols = 512;                      // two 256-column accumulators
 constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kStages * kStageBytes + 256 /*barriers*/;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
@@ -201,6 +212,11 @@ score_tiles_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&sh->tmem_base);
 
+    // Registers move from the control warpgroup (which needs few) to the two epilogue warpgroups
+    // (128 fp32 partial logits per thread): 128*120 + 256*184 <= 64K.  Each setmaxnreg sits at the
+    // top of the code it governs so that the register allocator sees which budget applies where.
+    if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 120;");
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -241,49 +257,56 @@ score_tiles_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_
         if (lane == 0) {
             constexpr uint32_t idesc = instr_desc_bf16(kBlockM, kBlockN);
             uint32_t stage = 0, phase = 0;
-            uint32_t tile_count = 0;
+            uint32_t chunk_count = 0;                        // accumulator hand-overs so far
             bool ok = true;
             for (int w = 0; w < plan.waves && ok; ++w) {
                 int mt, nb, ne;
                 if (!plan_unit(plan, w, cta, &mt, &nb, &ne)) continue;
-                for (int n = nb; n < ne && ok; ++n, ++tile_count) {
-                    const uint32_t buf = tile_count & 1u;
-                    const uint32_t use_phase = (tile_count >> 1) & 1u;
-                    if (!mbar_wait(smem_u32(&sh->acc_empty[buf]), use_phase ^ 1u, abort_flag, kWaitLimitNs, true)) {
-                        ok = false;
-                        break;
-                    }
-                    tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + buf * kBlockN;
-                    for (int kb = 0; kb < plan.k_blocks; ++kb) {
-                        if (!mbar_wait(smem_u32(&sh->full[stage]), phase, abort_flag, kWaitLimitNs, true)) {
+                for (int n = nb; n < ne && ok; ++n) {
+                    for (int kb0 = 0; kb0 < plan.k_blocks && ok; kb0 += plan.chunk_kblocks, ++chunk_count) {
+                        const uint32_t buf = chunk_count & 1u;
+                        const uint32_t use_phase = (chunk_count >> 1) & 1u;
+                        if (!mbar_wait(smem_u32(&sh->acc_empty[buf]), use_phase ^ 1u, abort_flag, kWaitLimitNs,
+                                       true)) {
                             ok = false;
                             break;
                         }
                         tc_fence_after();
-                        const uint32_t a_addr = tiles_addr + stage * kStageBytes;
-                        const uint64_t a_desc = smem_desc_k_major_sw128(a_addr);
-                        const uint64_t b_desc = smem_desc_k_major_sw128(a_addr + kABytes);
+                        const uint32_t d_tmem = tmem_base + buf * kBlockN;
+                        const int kb1 = min(kb0 + plan.chunk_kblocks, plan.k_blocks);
+                        for (int kb = kb0; kb < kb1; ++kb) {
+                            if (!mbar_wait(smem_u32(&sh->full[stage]), phase, abort_flag, kWaitLimitNs, true)) {
+                                ok = false;
+                                break;
+                            }
+                            tc_fence_after();
+                            const uint32_t a_addr = tiles_addr + stage * kStageBytes;
+                            const uint64_t a_desc = smem_desc_k_major_sw128(a_addr);
+                            const uint64_t b_desc = smem_desc_k_major_sw128(a_addr + kABytes);
 #pragma unroll
-                        for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-                            // advancing 16 bf16 (32 bytes) along K inside the swizzled row: +2 in the
-                            // 16-byte units of the descriptor's start-address field
-                            tc_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                        (kb | k) != 0 ? 1u : 0u);
+                            for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+                                // advancing 16 bf16 (32 bytes) along K inside the swizzled row: +2 in the
+                                // 16-byte units of the descriptor's start-address field
+                                tc_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                            (kb != kb0 || k != 0) ? 1u : 0u);
+                            }
+                            tc_commit(smem_u32(&sh->empty[stage]));   // frees the stage once these MMAs retire
+                            if (++stage == kStages) { stage = 0; phase ^= 1u; }
                         }
-                        tc_commit(smem_u32(&sh->empty[stage]));     // frees the stage once these MMAs retire
-                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                        if (ok) tc_commit(smem_u32(&sh->acc_full[buf]));  // chunk ready for the epilogue
                     }
-                    if (ok) tc_commit(smem_u32(&sh->acc_full[buf]));  // accumulator ready for the epilogue
                 }
             }
         }
+    }
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 184;");
+        // ------------------------------------------------------------------ epilogue (warps 4..11)
         const int quarter = warp & 3;                        // TMEM lanes 32*quarter .. +31 belong to this warp
+        const int half = (warp - 4) >> 2;                    // which 128 columns of the tile
         const int row_in_tile = quarter * 32 + lane;
         const uint32_t lane_field = static_cast<uint32_t>(quarter * 32) << 16;
-        uint32_t tile_count = 0;
+        uint32_t chunk_count = 0;
         bool ok = true;
         for (int w = 0; w < plan.waves && ok; ++w) {
             int mt, nb, ne;
@@ -292,50 +315,72 @@ score_tiles_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_
             const int32_t id = (row < plan.rows) ? token_ids[row] : -1;
             // state in base-2 units: run_max = max(z) * log2(e), run_sum = sum 2^(z*log2e - run_max)
             float run_max = -INFINITY, run_sum = 0.0f, picked = -INFINITY;
-            for (int n = nb; n < ne && ok; ++n, ++tile_count) {
-                const uint32_t buf = tile_count & 1u;
-                const uint32_t use_phase = (tile_count >> 1) & 1u;
-                if (!mbar_wait(smem_u32(&sh->acc_full[buf]), use_phase, abort_flag, kWaitLimitNs, true)) {
-                    ok = false;
-                    break;
+            for (int n = nb; n < ne && ok; ++n) {
+                float acc[kHalfN];                           // this thread's 128 logits of the tile
+                for (int kb0 = 0; kb0 < plan.k_blocks; kb0 += plan.chunk_kblocks, ++chunk_count) {
+                    const uint32_t buf = chunk_count & 1u;
+                    const uint32_t use_phase = (chunk_count >> 1) & 1u;
+                    if (!mbar_wait(smem_u32(&sh->acc_full[buf]), use_phase, abort_flag, kWaitLimitNs, true)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t taddr = tmem_base + lane_field + buf * kBlockN + half * kHalfN;
+                    if (kb0 == 0) {
+#pragma unroll
+                        for (int g = 0; g < kHalfN / 32; ++g) {
+                            float v[32];
+                            tmem_ld_32cols(taddr + g * 32, v);
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) acc[g * 32 + j] = v[j];
+                        }
+                    } else {
+#pragma unroll
+                        for (int g = 0; g < kHalfN / 32; ++g) {
+                            float v[32];
+                            tmem_ld_32cols(taddr + g * 32, v);
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) acc[g * 32 + j] += v[j];
+                        }
+                    }
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(&sh->acc_empty[buf]));   // the MMA issuer may reuse this buffer
                 }
-                tc_fence_after();
-                const int col_base = n * kBlockN;
-#pragma unroll 1
-                for (int c = 0; c < kBlockN / 32; ++c) {
-                    const int col0 = col_base + c * 32;
-                    const int valid = plan.V - col0;         // columns of this chunk inside the vocabulary
-                    if (valid <= 0) break;                   // uniform across the CTA
-                    float v[32];
-                    tmem_ld_32cols(tmem_base + lane_field + buf * kBlockN + c * 32, v);
-                    if (valid < 32) {
+                if (!ok) break;
+                const int col_base = n * kBlockN + half * kHalfN;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = (j < valid) ? v[j] : -INFINITY;
+                for (int g = 0; g < kHalfN / 32; ++g) {
+                    const int col0 = col_base + g * 32;
+                    const int valid = plan.V - col0;         // columns of this group inside the vocabulary
+                    if (valid > 0) {
+                        float* v = acc + g * 32;
+                        if (valid < 32) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] = (j < valid) ? v[j] : -INFINITY;
+                        }
+                        const uint32_t rel = static_cast<uint32_t>(id - col0);
+                        if (rel < 32u) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) picked = (rel == (uint32_t)j) ? v[j] : picked;
+                        }
+                        float cmax = v[0];
+#pragma unroll
+                        for (int j = 1; j < 32; ++j) cmax = fmaxf(cmax, v[j]);
+                        const float new_max = fmaxf(run_max, cmax * kLog2e);
+                        run_sum *= ex2_approx(run_max - new_max);  // 2^-inf = 0 on the first group
+                        run_max = new_max;
+                        float acc0 = 0.0f, acc1 = 0.0f;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 2) {
+                            acc0 += ex2_approx(fmaf(v[j], kLog2e, -new_max));
+                            acc1 += ex2_approx(fmaf(v[j + 1], kLog2e, -new_max));
+                        }
+                        run_sum += acc0 + acc1;
                     }
-                    const uint32_t rel = static_cast<uint32_t>(id - col0);
-                    if (rel < 32u) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) picked = (rel == (uint32_t)j) ? v[j] : picked;
-                    }
-                    float cmax = v[0];
-#pragma unroll
-                    for (int j = 1; j < 32; ++j) cmax = fmaxf(cmax, v[j]);
-                    const float new_max = fmaxf(run_max, cmax * kLog2e);
-                    run_sum *= ex2_approx(run_max - new_max);  // 2^-inf = 0 on the first chunk
-                    run_max = new_max;
-                    float acc0 = 0.0f, acc1 = 0.0f;
-#pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
-                        acc0 += ex2_approx(fmaf(v[j], kLog2e, -new_max));
-                        acc1 += ex2_approx(fmaf(v[j + 1], kLog2e, -new_max));
-                    }
-                    run_sum += acc0 + acc1;
                 }
-                tc_fence_before();
-                mbar_arrive(smem_u32(&sh->acc_empty[buf]));
             }
             if (ok) {
-                float* slot = workspace + ((size_t)w * plan.grid + cta) * kTripleFloats;
+                float* slot = workspace + ((size_t)w * plan.grid + cta) * kTripleFloats + half * 3 * kBlockM;
                 slot[row_in_tile] = run_max;
                 slot[kBlockM + row_in_tile] = run_sum;
                 slot[2 * kBlockM + row_in_tile] = picked;

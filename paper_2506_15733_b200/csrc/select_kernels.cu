@@ -16,9 +16,11 @@ constexpr double kLn2 = 0.6931471805599453094;
 constexpr unsigned kFull = 0xffffffffu;
 
 // ------------------------------------------------------------------------------------ merge
-// Workspace slot (wave * grid + cta) holds, for the 128 rows of that CTA's row tile, the running
-// maximum in base-2 units (max logit * log2 e), the sum of 2^(logit*log2e - max) over the CTA's
-// vocabulary chunk, and the drafted id's logit if the id fell into the chunk (-inf otherwise).
+// Workspace slot (wave * grid + cta) holds, for the 128 rows of that CTA's row tile and for each
+// half of the tile's 256 columns (the two epilogue threads of a row), the running maximum in
+// base-2 units (max logit * log2 e), the sum of 2^(logit*log2e - max) over that half of the CTA's
+// vocabulary chunk, and the drafted id's logit if the id fell there (-inf otherwise).  A half
+// that saw no valid column (vocabulary tail) carries max = -inf, sum = 0.
 __global__ void merge_splits_kernel(const ScorePlan plan, const float* __restrict__ workspace,
                                     const int32_t* __restrict__ token_ids, float* __restrict__ tok_logprob,
                                     uint32_t* __restrict__ status) {
@@ -33,14 +35,18 @@ __global__ void merge_splits_kernel(const ScorePlan plan, const float* __restric
     }
     const float* base = workspace + ((size_t)wave * plan.grid + i) * kTripleFloats + r;
     const size_t stride = (size_t)gm * kTripleFloats;       // next chunk of the same row tile
+    constexpr int kHalf = 3 * kBlockM;                      // second half of the tile's columns
     float gmax = -INFINITY;
-    for (int s = 0; s < splits; ++s) gmax = fmaxf(gmax, base[s * stride]);
+    for (int s = 0; s < splits; ++s) gmax = fmaxf(gmax, fmaxf(base[s * stride], base[s * stride + kHalf]));
     double sum = 0.0;
     float logit = -INFINITY;
     for (int s = 0; s < splits; ++s) {
-        const float* p = base + s * stride;
-        sum += (double)p[kBlockM] * exp2((double)p[0] - (double)gmax);
-        logit = fmaxf(logit, p[2 * kBlockM]);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const float* p = base + s * stride + h * kHalf;
+            if (p[0] != -INFINITY) sum += (double)p[kBlockM] * exp2((double)p[0] - (double)gmax);
+            logit = fmaxf(logit, p[2 * kBlockM]);
+        }
     }
     const int32_t id = token_ids[row];
     if (id < 0 || id >= plan.V) {

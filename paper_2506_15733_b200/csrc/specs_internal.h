@@ -17,7 +17,8 @@ namespace specs {
 constexpr int kBlockM = 128;   // drafted rows per tile   (= TMEM lanes, one epilogue thread per row)
 constexpr int kBlockN = 256;   // vocabulary entries per tile (= fp32 TMEM columns of one accumulator)
 constexpr int kBlockK = 64;    // bf16 elements per k-block: 128 bytes, one swizzle-128B row
-constexpr int kTripleFloats = 3 * kBlockM;   // one workspace slot: max[128], sumexp[128], logit[128]
+constexpr int kTripleFloats = 2 * 3 * kBlockM;   // one workspace slot: for each half of the 256 columns, max[128], sumexp[128], logit[128]
+constexpr int kDefaultChunkKBlocks = 8;      // k-blocks (of 64) per accumulation chunk: 512 elements of d
 
 // How the (row tile x vocab tile) grid is cut into persistent work units.
 //
@@ -40,10 +41,12 @@ struct ScorePlan {
     int32_t rem_m;         // row tiles of the last wave (0: none)
     int32_t split_rem;     // vocab chunks of the last wave
     int32_t waves;         // full_waves + (rem_m > 0)
+    int32_t chunk_kblocks; // k-blocks per fresh tensor-core accumulator (chunks are summed in registers)
 };
 
 // Host-side planner (pure arithmetic, no CUDA calls).
-ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms);
+ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms,
+                          int32_t chunk_kblocks = kDefaultChunkKBlocks);
 size_t plan_workspace_bytes(const ScorePlan& p);
 
 // Work unit of CTA `cta` in wave `wave`: returns false when the CTA idles in that wave.
@@ -73,6 +76,7 @@ struct specs_ctx {
     int device = 0;
     int num_sms = 0;
     int engine = SPECS_ENGINE_TCGEN05;
+    int chunk_kblocks = specs::kDefaultChunkKBlocks;   // see specs_set_accum_chunk
     uint32_t* d_status = nullptr;          // device status word (SPECS_DEV_* bits)
     specs::EncodeTiledFn encode_tiled = nullptr;
     // grow-only device arena for specs_beam_step_host

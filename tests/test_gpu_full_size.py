@@ -1,0 +1,169 @@
+"""GPU parity at the full benchmark sizes, in the launch configuration bench.py times.
+
+The CUDA path scores every row; the CPU oracle scores a seeded sample of whole blocks (plus
+single rows, e.g. the outlier rows of the stress config) -- rows are independent, so a sample is
+exact for parity.  Selection is checked two ways and labelled: end to end on problems whose blocks
+were all scored by the oracle, and "selection logic" on all problems by handing the GPU's block
+log-probabilities to the oracle's scoring / sampling / switch functions.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import specs_oracle as O
+from paper_2506_15733_b200 import binding
+from paper_2506_15733_b200 import inputs as I
+from tests.gpu_util import BLK_RTOL, MARGIN, TOK_ATOL, DeviceStep
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(0)
+    yield c
+    assert c.device_status() == 0
+    c.close()
+
+
+def rows_of_blocks(x, blocks):
+    return np.concatenate([np.arange(x.block_offsets[b], x.block_offsets[b + 1]) for b in blocks]).astype(np.int64)
+
+
+def check_sampled_rows(x, got_tok, rows_idx, w_f64):
+    want = O.token_logprobs(x.hidden[rows_idx], x.w_vocab, x.token_ids[rows_idx], w_f64=w_f64)
+    err = np.abs(got_tok[rows_idx] - want)
+    assert np.all(np.isfinite(got_tok)), "non-finite token log-prob somewhere in the full output"
+    assert err.max() <= TOK_ATOL, f"token log-prob off by {err.max():.3e} (row {rows_idx[int(err.argmax())]})"
+    return want, float(err.max())
+
+
+def check_block_sums(x, got, blocks, want_tok_by_row):
+    for b in blocks:
+        a, e = int(x.block_offsets[b]), int(x.block_offsets[b + 1])
+        want = O.block_sums(np.array([want_tok_by_row[t] for t in range(a, e)]), np.array([0, e - a]))[0]
+        for key in ("blk_logprob", "blk_logprob_f64"):
+            assert abs(got[key][b] - want) <= BLK_RTOL * abs(want), (key, b, got[key][b], want)
+    # every block sum on the GPU equals the plain sum of the GPU's own token log-probs (all blocks)
+    all_sums = O.block_sums(got["tok_logprob"], x.block_offsets)
+    assert np.allclose(got["blk_logprob_f64"], all_sums, rtol=1e-12, atol=1e-9)
+
+
+def check_selection_logic(x, got, beta, tau, gen_blk):
+    """Oracle O4-O7 on the GPU's own block log-probs: picks exact above the margin, weights, flags."""
+    S = O.scores(got["blk_logprob_f64"], gen_blk, x.reward, beta)
+    want_c, margin = O.gumbel_pick(S, x.uniforms, x.cand_offsets)
+    sure = margin > MARGIN
+    assert np.array_equal(got["chosen"][sure], want_c[sure])
+    assert np.abs(got["weights"] - O.weights(S, x.cand_offsets)).max() < 1e-6
+    assert np.array_equal(got["accept"], O.accept_flags(x.reward, x.cand_offsets, tau))
+    return int(sure.sum())
+
+
+def test_step7b_all_rows_all_betas(ctx):
+    cfg = I.CONFIGS["step7b"]
+    x = I.make_step_inputs(cfg)
+    s = DeviceStep(ctx, x)
+    got = s.step(cfg.betas[0], 0.7)
+    w64 = O.bf16_bits_to_f64(x.w_vocab)
+    all_rows = np.arange(x.rows)
+    want_tok, err = check_sampled_rows(x, got["tok_logprob"], all_rows, w64)
+    check_block_sums(x, got, range(x.blocks), want_tok)
+    LP = O.block_sums(want_tok, x.block_offsets)
+    LQ = O.block_sums(x.draft_tok_logprob, x.block_offsets)
+    assert np.allclose(got["blk_logprob_gen"], LQ, rtol=1e-12)
+    for beta in cfg.betas:
+        s.select(beta, 0.7)
+        torch.cuda.synchronize()
+        g = s.results()
+        # end to end: oracle block log-probs vs GPU block log-probs
+        S = O.scores(LP, LQ, x.reward, beta)
+        want_c, margin = O.gumbel_pick(S, x.uniforms, x.cand_offsets)
+        slack = 2 * np.abs(g["blk_logprob_f64"] - LP).max()
+        if margin[0] > MARGIN + slack:
+            assert g["chosen"][0] == want_c[0]
+        assert np.abs(g["weights"] - O.weights(S, x.cand_offsets)).max() < 5e-3 + 2 * slack
+        check_selection_logic(x, g, beta, 0.7, LQ)
+
+
+def test_batched_ragged_step(ctx):
+    cfg = I.CONFIGS["batched"]
+    x = I.make_step_inputs(cfg)
+    assert x.rows == 20893
+    s = DeviceStep(ctx, x)
+    got = s.step(2.0, cfg.taus[0])
+    w64 = O.bf16_bits_to_f64(x.w_vocab)
+    rng = np.random.Generator(np.random.Philox(key=[7002, 1]))
+    blocks = list(range(8)) + sorted(rng.choice(np.arange(8, 256), size=4, replace=False).tolist())   # problem 0 whole
+    rows_idx = rows_of_blocks(x, blocks)
+    want_tok, err = check_sampled_rows(x, got["tok_logprob"], rows_idx, w64)
+    by_row = dict(zip(rows_idx.tolist(), want_tok.tolist()))
+    check_block_sums(x, got, blocks, by_row)
+    LQ = O.block_sums(x.draft_tok_logprob, x.block_offsets)
+    # end to end on problem 0
+    LP0 = np.array([sum(by_row[t] for t in range(x.block_offsets[b], x.block_offsets[b + 1])) for b in range(8)])
+    S0 = O.scores(LP0, LQ[:8], x.reward[:8], 2.0)
+    c0, m0 = O.gumbel_pick(S0, x.uniforms[:8], np.array([0, 8]))
+    slack = 2 * np.abs(got["blk_logprob_f64"][:8] - LP0).max()
+    if m0[0] > MARGIN + slack:
+        assert got["chosen"][0] == c0[0]
+    # selection logic on all 32 problems, and the threshold sweep
+    for tau in cfg.taus:
+        s.select(2.0, tau)
+        torch.cuda.synchronize()
+        assert check_selection_logic(x, s.results(), 2.0, tau, LQ) >= 24
+
+
+@pytest.mark.parametrize("token_dist", ["zipf", "zipf_perm"])
+def test_dual_scoring_draft_then_target(ctx, token_dist):
+    # the same 65536 drafted tokens scored with a 1.5B-draft-shaped head and a 7B-target-shaped head;
+    # the draft pass supplies the generator's block log-probs (Eq. 1's denominator)
+    rng = np.random.Generator(np.random.Philox(key=[7003, 1]))
+    blocks = sorted(rng.choice(256, size=3, replace=False).tolist())
+    blk = {}
+    for name in ("dual_draft", "dual_target"):
+        cfg = I.scaled(I.CONFIGS[name], token_dist=token_dist)
+        x = I.make_step_inputs(cfg)
+        s = DeviceStep(ctx, x)
+        s.score()
+        torch.cuda.synchronize()
+        got = s.results()
+        w64 = O.bf16_bits_to_f64(x.w_vocab)
+        rows_idx = np.unique(np.concatenate([rows_of_blocks(x, blocks), rng.choice(x.rows, 128, replace=False)]))
+        want_tok, err = check_sampled_rows(x, got["tok_logprob"], rows_idx, w64)
+        check_block_sums(x, got, blocks, dict(zip(rows_idx.tolist(), want_tok.tolist())))
+        blk[name] = s.blk_lp64.clone()
+        keep = s
+        del w64
+    # selection with LP from the target pass and LQ from the draft pass, on the last pass's buffers
+    keep.ctx.specs_subsample(blk["dual_target"], blk["dual_draft"], keep.reward, keep.cand_offsets, 1.0,
+                             keep.uniforms, keep.chosen, keep.weights, 0.7, keep.accept)
+    torch.cuda.synchronize()
+    g = keep.results()
+    g["blk_logprob_f64"] = blk["dual_target"].cpu().numpy()
+    assert check_selection_logic(x, g, 1.0, 0.7, blk["dual_draft"].cpu().numpy()) >= 6
+
+
+def test_stress_heavy_tailed_logits(ctx):
+    cfg = I.CONFIGS["stress"]
+    x = I.make_step_inputs(cfg)
+    s = DeviceStep(ctx, x)
+    got = s.step(cfg.betas[0], 0.7)
+    w64 = O.bf16_bits_to_f64(x.w_vocab)
+    rng = np.random.Generator(np.random.Philox(key=[7004, 1]))
+    # blocks that contain outlier rows (shortest three of them), 160 outlier rows, 64 ordinary rows
+    blk_of_row = np.searchsorted(x.block_offsets, x.outlier_rows, side="right") - 1
+    cand_blocks = np.unique(blk_of_row)
+    lens = np.diff(x.block_offsets)[cand_blocks]
+    blocks = cand_blocks[np.argsort(lens)[:3]].tolist()
+    rows_idx = np.unique(np.concatenate([rows_of_blocks(x, blocks),
+                                         rng.choice(x.outlier_rows, 160, replace=False),
+                                         rng.choice(x.rows, 64, replace=False)]))
+    want_tok, err = check_sampled_rows(x, got["tok_logprob"], rows_idx, w64)
+    assert np.abs(want_tok).max() > 100                       # the sample really holds heavy-tailed rows
+    check_block_sums(x, got, blocks, dict(zip(rows_idx.tolist(), want_tok.tolist())))
+    LQ = O.block_sums(x.draft_tok_logprob, x.block_offsets)
+    for beta in cfg.betas:
+        s.select(beta, 0.7)
+        torch.cuda.synchronize()
+        check_selection_logic(x, s.results(), beta, 0.7, LQ)

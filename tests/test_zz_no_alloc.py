@@ -79,7 +79,7 @@ def test_noalloc_reports_bad_ids_and_rejects_oversized_problems():
     # a plan that needs more scratch than the fixed array: refused on the host, nothing launched.
     # Only the shapes matter for the refusal, so the tensors below are never read.
     sms = torch.cuda.get_device_properties(0).multi_processor_count
-    rows = 128 * sms * 20                                     # 20 full waves at d = 64 -> 20 * sms * 1536 bytes
+    rows = 128 * sms * 20                                     # 20 full waves at d = 64 -> 20 * sms * 3072 bytes
     assert binding.score_plan(rows, 64, 300, sms)["workspace_bytes"] > binding.NOALLOC_SCRATCH_BYTES
     big_h = torch.empty((rows, 64), dtype=torch.bfloat16, device="cuda:0")
     big_ids = torch.zeros(rows, dtype=torch.int32, device="cuda:0")
