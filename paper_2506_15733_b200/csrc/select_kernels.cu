@@ -21,12 +21,21 @@ constexpr unsigned kFull = 0xffffffffu;
 // base-2 units (max logit * log2 e), the sum of 2^(logit*log2e - max) over that half of the CTA's
 // vocabulary chunk, and the drafted id's logit if the id fell there (-inf otherwise).  A half
 // that saw no valid column (vocabulary tail) carries max = -inf, sum = 0.
-__global__ void merge_splits_kernel(const ScorePlan plan, const float* __restrict__ workspace,
-                                    const int32_t* __restrict__ token_ids, float* __restrict__ tok_logprob,
-                                    uint32_t* __restrict__ status) {
-    const int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (row >= plan.rows) return;
-    const int mt = (int)(row / kBlockM), r = (int)(row % kBlockM);
+constexpr int kMergeWarps = 8;                              // warps per block: each takes every 8th split
+
+__global__ void __launch_bounds__(32 * kMergeWarps)
+merge_splits_kernel(const ScorePlan plan, const float* __restrict__ workspace,
+                    const int32_t* __restrict__ token_ids, float* __restrict__ tok_logprob,
+                    uint32_t* __restrict__ status) {
+    // A block owns 32 consecutive rows (lane = row, so loads are coalesced); its warps share the
+    // vocabulary splits of those rows and combine their partial (max, sum, logit) in shared memory.
+    __shared__ float sh_max[kMergeWarps][32], sh_logit[kMergeWarps][32];
+    __shared__ double sh_sum[kMergeWarps][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t row = (int64_t)blockIdx.x * 32 + lane;
+    const bool live = row < plan.rows;
+    const int64_t row_c = live ? row : plan.rows - 1;
+    const int mt = (int)(row_c / kBlockM), r = (int)(row_c % kBlockM);
     int wave, i, gm, splits;
     if (mt < plan.full_waves * plan.group_m) {
         wave = mt / plan.group_m; i = mt % plan.group_m; gm = plan.group_m; splits = plan.split_full;
@@ -36,17 +45,34 @@ __global__ void merge_splits_kernel(const ScorePlan plan, const float* __restric
     const float* base = workspace + ((size_t)wave * plan.grid + i) * kTripleFloats + r;
     const size_t stride = (size_t)gm * kTripleFloats;       // next chunk of the same row tile
     constexpr int kHalf = 3 * kBlockM;                      // second half of the tile's columns
-    float gmax = -INFINITY;
-    for (int s = 0; s < splits; ++s) gmax = fmaxf(gmax, fmaxf(base[s * stride], base[s * stride + kHalf]));
+
+    float m = -INFINITY, logit = -INFINITY;
     double sum = 0.0;
-    float logit = -INFINITY;
-    for (int s = 0; s < splits; ++s) {
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const float* p = base + s * stride + h * kHalf;
-            if (p[0] != -INFINITY) sum += (double)p[kBlockM] * exp2((double)p[0] - (double)gmax);
-            logit = fmaxf(logit, p[2 * kBlockM]);
+    for (int s = warp; s < splits; s += kMergeWarps) {
+        const float* p = base + s * stride;
+        const float m0 = p[0], s0 = p[kBlockM], t0 = p[2 * kBlockM];
+        const float m1 = p[kHalf], s1 = p[kHalf + kBlockM], t1 = p[kHalf + 2 * kBlockM];
+        const float mn = fmaxf(m, fmaxf(m0, m1));
+        if (mn != -INFINITY) {
+            // exp2f(-inf) = 0 takes care of halves and states that have seen nothing yet
+            sum = sum * (double)exp2f(m - mn) + (double)s0 * (double)exp2f(m0 - mn) +
+                  (double)s1 * (double)exp2f(m1 - mn);
+            m = mn;
         }
+        logit = fmaxf(logit, fmaxf(t0, t1));
+    }
+    sh_max[warp][lane] = m; sh_sum[warp][lane] = sum; sh_logit[warp][lane] = logit;
+    __syncthreads();
+    if (warp != 0 || !live) return;
+    float gmax = sh_max[0][lane];
+#pragma unroll
+    for (int w = 1; w < kMergeWarps; ++w) gmax = fmaxf(gmax, sh_max[w][lane]);
+    double total = 0.0;
+    float picked = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kMergeWarps; ++w) {
+        if (sh_max[w][lane] != -INFINITY) total += sh_sum[w][lane] * (double)exp2f(sh_max[w][lane] - gmax);
+        picked = fmaxf(picked, sh_logit[w][lane]);
     }
     const int32_t id = token_ids[row];
     if (id < 0 || id >= plan.V) {
@@ -54,8 +80,8 @@ __global__ void merge_splits_kernel(const ScorePlan plan, const float* __restric
         atomicOr(status, SPECS_DEV_TOKEN_RANGE);
         return;
     }
-    const double lse = ((double)gmax + log2(sum)) * kLn2;   // natural-log normaliser
-    tok_logprob[row] = (float)((double)logit - lse);
+    const double lse = ((double)gmax + log2(total)) * kLn2; // natural-log normaliser
+    tok_logprob[row] = (float)((double)picked - lse);
 }
 
 // ------------------------------------------------------------------------------------ block sums
@@ -160,9 +186,9 @@ inline unsigned warps_grid(int64_t warps, int threads) {
 int launch_merge(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, const int32_t* token_ids,
                  float* tok_logprob, cudaStream_t stream) {
     if (plan.rows == 0) return SPECS_OK;
-    const int threads = 128;
-    const unsigned blocks = (unsigned)((plan.rows + threads - 1) / threads);
-    merge_splits_kernel<<<blocks, threads, 0, stream>>>(plan, workspace, token_ids, tok_logprob, ctx->d_status);
+    const unsigned blocks = (unsigned)((plan.rows + 31) / 32);
+    merge_splits_kernel<<<blocks, 32 * kMergeWarps, 0, stream>>>(plan, workspace, token_ids, tok_logprob,
+                                                                 ctx->d_status);
     return cuda_status(cudaGetLastError());
 }
 
