@@ -55,8 +55,12 @@ typedef enum specs_status {
 #define SPECS_DEV_TOKEN_RANGE  0x2u
 
 /* Scoring engines (see specs_set_engine). */
-#define SPECS_ENGINE_TCGEN05 0   /* tensor-core path: TMA + tcgen05.mma + TMEM, fused epilogue (default) */
-#define SPECS_ENGINE_SIMT    1   /* plain CUDA-core kernel; a bring-up and bisecting aid, never chosen automatically */
+#define SPECS_ENGINE_TCGEN05      0   /* tensor-core path: TMA + tcgen05.mma + TMEM, fused epilogue (default);
+                                        the planner picks the tile shape (one CTA or a CTA pair per tile) */
+#define SPECS_ENGINE_SIMT         1   /* plain CUDA-core kernel; a bring-up and bisecting aid, never chosen automatically */
+#define SPECS_ENGINE_TCGEN05_1CTA 2   /* tensor-core path, forced to 128-row tiles run by single CTAs */
+#define SPECS_ENGINE_TCGEN05_2CTA 3   /* tensor-core path, forced to 256-row tiles run by CTA pairs
+                                        (tcgen05.mma.cta_group::2; each CTA stages half of the W tile) */
 
 /* Human-readable name of a status value (static string, never NULL). */
 const char* specs_status_string(int status);
@@ -67,7 +71,9 @@ const char* specs_status_string(int status);
 int specs_create(specs_ctx** out, int device);
 int specs_destroy(specs_ctx* ctx);
 
-/* Select the scoring engine for later specs_score_blocks calls on this context. */
+/* Select the scoring engine for later specs_score_blocks calls on this context
+ * (SPECS_ERR_SHAPE for an unknown value; SPECS_ERR_CUDA if CTA pairs were asked
+ * for and the device cannot launch them). */
 int specs_set_engine(specs_ctx* ctx, int engine);
 
 /* Length, in elements of d, of one tensor-core accumulation chunk (a multiple of
@@ -78,7 +84,8 @@ int specs_set_engine(specs_ctx* ctx, int engine);
  * which divides the bias by the number of chunks.  Shorter chunks cost epilogue time. */
 int specs_set_accum_chunk(specs_ctx* ctx, int32_t k_elements);
 
-/* Number of SMs the context schedules over (also the persistent grid size). */
+/* Number of SMs the context schedules over (the persistent grid is one CTA per SM,
+ * or two per resident CTA pair). */
 int specs_sm_count(const specs_ctx* ctx);
 
 /* Bytes of scratch specs_score_blocks needs for these sizes.  It holds one
@@ -193,18 +200,23 @@ int   specs_set_timing(specs_ctx* ctx, int enabled);
 float specs_score_kernel_ms(specs_ctx* ctx, int32_t* h_launches);
 
 /* The work-unit plan of the tensor-core scoring kernel, for inspection and tests
- * (pure host arithmetic, needs no device).  The row tiles (128 rows) x vocabulary
- * tiles (256 entries) grid is processed in waves; in a wave, gm row tiles are live
- * and the vocabulary is cut into s contiguous chunks, one persistent CTA per
- * (row tile, chunk).  h_out12 receives: row_tiles, vocab_tiles, k_blocks, grid,
- * group_m, split_full, full_waves, rem_m, split_rem, waves, and the workspace size
- * in bytes as two 31-bit halves (low, high). */
-int specs_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t* h_out12);
+ * (pure host arithmetic, needs no device).  A work unit is one CTA (cta_group 1,
+ * a 128-row super tile) or a pair of CTAs of one cluster (cta_group 2, a 256-row
+ * super tile); cta_group 0 lets the planner choose as the default engine does,
+ * assuming num_sms / 2 resident pairs.  The super tiles x vocabulary tiles (256
+ * entries) grid is processed in waves; in a wave, gm super tiles are live and the
+ * vocabulary is cut into s contiguous chunks, one persistent unit per (super tile,
+ * chunk).  h_out16 receives: row_tiles, vocab_tiles, k_blocks, grid (CTAs), group_m,
+ * split_full, full_waves, rem_m, split_rem, waves, the workspace size in bytes as
+ * two 31-bit halves (low, high), cta_group, units per wave, super_tiles, and the
+ * k-blocks per accumulation chunk. */
+int specs_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t cta_group, int32_t* h_out16);
 
-/* Work unit of CTA `cta` in wave `wave` under that plan: h_out3 = {row tile,
- * first vocab tile, one-past-last vocab tile}; row tile -1 when the CTA idles. */
-int specs_score_plan_unit(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t wave, int32_t cta,
-                          int32_t* h_out3);
+/* Work of CTA `cta` in wave `wave` under that plan: h_out3 = {its 128-row tile,
+ * first vocab tile, one-past-last vocab tile}; row tile -1 when the CTA has no
+ * rows in that wave (idle unit, or the second CTA of a pair past the last tile). */
+int specs_score_plan_unit(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t cta_group, int32_t wave,
+                          int32_t cta, int32_t* h_out3);
 
 /* Block scoring for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this entry point exists for deployment, not for the method.)

@@ -20,6 +20,8 @@ _lib = None
 OK = 0
 ENGINE_TCGEN05 = 0
 ENGINE_SIMT = 1
+ENGINE_TCGEN05_1CTA = 2
+ENGINE_TCGEN05_2CTA = 3
 DEV_TIMEOUT = 0x1
 DEV_TOKEN_RANGE = 0x2
 
@@ -46,8 +48,8 @@ SIGNATURES = {
     "specs_set_timing": (C.c_int, [_vp, C.c_int]),
     "specs_score_kernel_ms": (C.c_float, [_vp, C.POINTER(_i32)]),
     "specs_score_blocks_noalloc": (C.c_int, [_vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]),
-    "specs_score_plan": (C.c_int, [_i64, _i32, _i32, _i32, C.POINTER(_i32)]),
-    "specs_score_plan_unit": (C.c_int, [_i64, _i32, _i32, _i32, _i32, _i32, C.POINTER(_i32)]),
+    "specs_score_plan": (C.c_int, [_i64, _i32, _i32, _i32, _i32, C.POINTER(_i32)]),
+    "specs_score_plan_unit": (C.c_int, [_i64, _i32, _i32, _i32, _i32, _i32, _i32, C.POINTER(_i32)]),
 }
 
 
@@ -97,19 +99,21 @@ def _stream() -> Optional[int]:
     return torch.cuda.current_stream().cuda_stream or None
 
 
-def score_plan(rows: int, d: int, V: int, num_sms: int) -> dict:
-    out = (_i32 * 12)()
-    _check(load_library().specs_score_plan(rows, d, V, num_sms, out), "specs_score_plan")
+def score_plan(rows: int, d: int, V: int, num_sms: int, cta_group: int = 0) -> dict:
+    out = (_i32 * 16)()
+    _check(load_library().specs_score_plan(rows, d, V, num_sms, cta_group, out), "specs_score_plan")
     keys = ["row_tiles", "vocab_tiles", "k_blocks", "grid", "group_m", "split_full", "full_waves", "rem_m",
             "split_rem", "waves"]
     plan = {k: int(out[i]) for i, k in enumerate(keys)}
     plan["workspace_bytes"] = int(out[10]) + (int(out[11]) << 31)
+    plan.update(cta_group=int(out[12]), units=int(out[13]), super_tiles=int(out[14]), chunk_kblocks=int(out[15]))
     return plan
 
 
-def score_plan_unit(rows: int, d: int, V: int, num_sms: int, wave: int, cta: int):
+def score_plan_unit(rows: int, d: int, V: int, num_sms: int, wave: int, cta: int, cta_group: int = 0):
     out = (_i32 * 3)()
-    _check(load_library().specs_score_plan_unit(rows, d, V, num_sms, wave, cta, out), "specs_score_plan_unit")
+    _check(load_library().specs_score_plan_unit(rows, d, V, num_sms, cta_group, wave, cta, out),
+           "specs_score_plan_unit")
     return int(out[0]), int(out[1]), int(out[2])
 
 

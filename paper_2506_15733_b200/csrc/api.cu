@@ -9,42 +9,78 @@
 namespace specs {
 
 // ---------------------------------------------------------------------------------- planner
-ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t chunk_kblocks) {
+namespace {
+
+// Estimated duration of a plan, in seconds: per wave, the busiest unit's run of vocabulary
+// tiles at the tensor rate the kernel reaches, or the HBM time of streaming W once, whichever
+// is longer.  The constants only rank candidate plans; they are not performance claims.
+constexpr double kPlanClockHz = 1.4e9;            // SM clock under sustained tensor load
+constexpr double kPlanHbmBytesPerS = 6.0e12;
+constexpr double kPlanL2Budget = 50.0e6;          // bytes of hidden-state tiles kept live per wave
+constexpr double kPlanTensorEff1 = 0.76;          // one CTA per unit: bounded by L2 -> SM operand delivery
+constexpr double kPlanTensorEff2 = 0.93;          // CTA pair: each CTA stages only half of the W tile
+
+double fill_plan(ScorePlan* p, int32_t cta_group, int32_t units) {
+    p->cta_group = cta_group;
+    p->units = units;
+    p->grid = units * cta_group;
+    p->super_tiles = (p->row_tiles + cta_group - 1) / cta_group;
+    const double tile_bytes = (double)kBlockM * cta_group * p->d * 2.0;
+    const double t_tile = (double)p->k_blocks * 512.0 / (cta_group == 2 ? kPlanTensorEff2 : kPlanTensorEff1) /
+                          kPlanClockHz;
+    const double w_bytes = (double)p->V * p->d * 2.0;
+    auto wave_time = [&](int gm, int s) {
+        const int run = (p->vocab_tiles + s - 1) / s;          // vocabulary tiles of the busiest unit
+        const double t_hbm = (w_bytes + gm * tile_bytes) / kPlanHbmBytesPerS;
+        const double t_mma = run * t_tile;
+        return t_mma > t_hbm ? t_mma : t_hbm;
+    };
+    double best = -1.0;
+    const int s_max = units < p->vocab_tiles ? units : p->vocab_tiles;
+    for (int s = 1; s <= s_max; ++s) {
+        const int gm = units / s;
+        if (gm > 1 && gm * tile_bytes > kPlanL2Budget) continue;
+        const int full = p->super_tiles / gm;
+        const int rem = p->super_tiles - full * gm;
+        int s_rem = 0;
+        double cost = full * wave_time(gm, s);
+        if (rem > 0) {
+            s_rem = units / rem;
+            if (s_rem > p->vocab_tiles) s_rem = p->vocab_tiles;
+            if (s_rem < 1) s_rem = 1;
+            cost += wave_time(rem, s_rem);
+        }
+        if (best < 0.0 || cost < best * (1.0 - 1e-9)) {
+            best = cost;
+            p->group_m = gm; p->split_full = s; p->full_waves = full; p->rem_m = rem; p->split_rem = s_rem;
+        }
+    }
+    p->waves = p->full_waves + (p->rem_m > 0 ? 1 : 0);
+    return best;
+}
+
+}  // namespace
+
+ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t pair_units,
+                          int32_t cta_group, int32_t chunk_kblocks) {
     ScorePlan p;
     std::memset(&p, 0, sizeof(p));
     p.rows = rows; p.d = d; p.V = V;
     p.row_tiles = (int32_t)((rows + kBlockM - 1) / kBlockM);
     p.vocab_tiles = (V + kBlockN - 1) / kBlockN;
     p.k_blocks = (d + kBlockK - 1) / kBlockK;
-    p.grid = num_sms;
     p.chunk_kblocks = (chunk_kblocks > 0 && chunk_kblocks < p.k_blocks) ? chunk_kblocks : p.k_blocks;
-    if (p.row_tiles == 0) return p;
-
-    // Full waves: the fewest vocabulary chunks s (hence the most row tiles gm = grid / s sharing
-    // each streamed W tile) such that the wave's hidden tiles stay well inside L2 and at most 2%
-    // of the CTAs idle.
-    const double tile_bytes = (double)kBlockM * d * 2.0;
-    const double l2_budget = 50.0e6;
-    int best_s = num_sms;                     // gm = 1 always fits
-    for (int s = 1; s <= num_sms; ++s) {
-        const int gm = num_sms / s;
-        if (gm * tile_bytes > l2_budget && gm > 1) continue;
-        if ((double)(gm * s) < 0.98 * num_sms) continue;
-        best_s = s;
-        break;
+    if (pair_units <= 0 && cta_group == 2) cta_group = 1;      // pairs unavailable on this device
+    if (cta_group == 1 || pair_units <= 0) {
+        fill_plan(&p, 1, num_sms);
+    } else if (cta_group == 2) {
+        fill_plan(&p, 2, pair_units);
+    } else {
+        ScorePlan q = p;
+        const double c1 = fill_plan(&p, 1, num_sms);
+        const double c2 = fill_plan(&q, 2, pair_units);
+        if (c2 < c1) p = q;
     }
-    if (best_s > p.vocab_tiles) best_s = p.vocab_tiles;       // a chunk holds at least one vocab tile
-    p.split_full = best_s;
-    p.group_m = num_sms / best_s;
-    p.full_waves = p.row_tiles / p.group_m;
-    p.rem_m = p.row_tiles - p.full_waves * p.group_m;
-    if (p.rem_m > 0) {
-        int s = num_sms / p.rem_m;
-        if (s > p.vocab_tiles) s = p.vocab_tiles;
-        if (s < 1) s = 1;
-        p.split_rem = s;
-    }
-    p.waves = p.full_waves + (p.rem_m > 0 ? 1 : 0);
     return p;
 }
 
@@ -145,6 +181,7 @@ int specs_create(specs_ctx** out, int device) {
         delete ctx;
         return SPECS_ERR_CUDA;
     }
+    ctx->pair_units = query_pair_units(device, ctx->num_sms);
     *out = ctx;
     return SPECS_OK;
 }
@@ -161,7 +198,10 @@ int specs_destroy(specs_ctx* ctx) {
 
 int specs_set_engine(specs_ctx* ctx, int engine) {
     if (!ctx) return SPECS_ERR_NULL;
-    if (engine != SPECS_ENGINE_TCGEN05 && engine != SPECS_ENGINE_SIMT) return SPECS_ERR_SHAPE;
+    if (engine != SPECS_ENGINE_TCGEN05 && engine != SPECS_ENGINE_SIMT && engine != SPECS_ENGINE_TCGEN05_1CTA &&
+        engine != SPECS_ENGINE_TCGEN05_2CTA)
+        return SPECS_ERR_SHAPE;
+    if (engine == SPECS_ENGINE_TCGEN05_2CTA && ctx->pair_units <= 0) return SPECS_ERR_CUDA;
     ctx->engine = engine;
     return SPECS_OK;
 }
@@ -177,30 +217,39 @@ int specs_sm_count(const specs_ctx* ctx) { return ctx ? ctx->num_sms : 0; }
 
 size_t specs_score_workspace_bytes(const specs_ctx* ctx, int64_t rows, int32_t d, int32_t V) {
     if (!ctx || check_score_shapes(rows, d, V, 0) != SPECS_OK) return 0;
-    return plan_workspace_bytes(make_score_plan(rows, d, V, ctx->num_sms));
+    // enough for whichever tile shape the engine setting selects at call time
+    const size_t one = plan_workspace_bytes(make_score_plan(rows, d, V, ctx->num_sms, ctx->pair_units, 1));
+    const size_t two = plan_workspace_bytes(make_score_plan(rows, d, V, ctx->num_sms, ctx->pair_units, 2));
+    return one > two ? one : two;
 }
 
-int specs_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t* h_out12) {
-    if (!h_out12) return SPECS_ERR_NULL;
-    if (check_score_shapes(rows, d, V, 0) != SPECS_OK || num_sms <= 0) return SPECS_ERR_SHAPE;
-    const ScorePlan p = make_score_plan(rows, d, V, num_sms);
-    const int32_t v[12] = {p.row_tiles, p.vocab_tiles, p.k_blocks, p.grid, p.group_m, p.split_full,
+int specs_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t cta_group, int32_t* h_out16) {
+    if (!h_out16) return SPECS_ERR_NULL;
+    if (check_score_shapes(rows, d, V, 0) != SPECS_OK || num_sms <= 0 || cta_group < 0 || cta_group > 2)
+        return SPECS_ERR_SHAPE;
+    const ScorePlan p = make_score_plan(rows, d, V, num_sms, num_sms / 2, cta_group);
+    const size_t ws = plan_workspace_bytes(p);
+    const int32_t v[16] = {p.row_tiles, p.vocab_tiles, p.k_blocks, p.grid, p.group_m, p.split_full,
                            p.full_waves, p.rem_m, p.split_rem, p.waves,
-                           (int32_t)(plan_workspace_bytes(p) & 0x7fffffff), (int32_t)(plan_workspace_bytes(p) >> 31)};
-    std::memcpy(h_out12, v, sizeof(v));
+                           (int32_t)(ws & 0x7fffffff), (int32_t)(ws >> 31),
+                           p.cta_group, p.units, p.super_tiles, p.chunk_kblocks};
+    std::memcpy(h_out16, v, sizeof(v));
     return SPECS_OK;
 }
 
-int specs_score_plan_unit(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t wave, int32_t cta,
-                          int32_t* h_out3) {
+int specs_score_plan_unit(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t cta_group, int32_t wave,
+                          int32_t cta, int32_t* h_out3) {
     if (!h_out3) return SPECS_ERR_NULL;
-    if (check_score_shapes(rows, d, V, 0) != SPECS_OK || num_sms <= 0) return SPECS_ERR_SHAPE;
-    const ScorePlan p = make_score_plan(rows, d, V, num_sms);
-    int mt = -1, nb = 0, ne = 0;
-    if (wave < 0 || wave >= p.waves || cta < 0 || cta >= p.grid || !plan_unit(p, wave, cta, &mt, &nb, &ne)) {
-        h_out3[0] = -1; h_out3[1] = 0; h_out3[2] = 0;
+    if (check_score_shapes(rows, d, V, 0) != SPECS_OK || num_sms <= 0 || cta_group < 0 || cta_group > 2)
+        return SPECS_ERR_SHAPE;
+    const ScorePlan p = make_score_plan(rows, d, V, num_sms, num_sms / 2, cta_group);
+    int st = -1, nb = 0, ne = 0;
+    h_out3[0] = -1; h_out3[1] = 0; h_out3[2] = 0;
+    if (wave < 0 || wave >= p.waves || cta < 0 || cta >= p.grid ||
+        !plan_unit(p, wave, cta / p.cta_group, &st, &nb, &ne))
         return SPECS_OK;
-    }
+    const int mt = st * p.cta_group + cta % p.cta_group;     // the CTA's own 128-row tile
+    if (mt >= p.row_tiles) return SPECS_OK;                  // second CTA of a pair past the last row tile
     h_out3[0] = mt; h_out3[1] = nb; h_out3[2] = ne;
     return SPECS_OK;
 }
@@ -224,7 +273,10 @@ int specs_score_blocks(specs_ctx* ctx, const void* hidden, const void* W_vocab, 
             st = launch_score_simt(ctx, hidden, W_vocab, token_ids, rows, d, V, tok_logprob, stream);
             if (st != SPECS_OK) return st;
         } else {
-            const ScorePlan plan = make_score_plan(rows, d, V, ctx->num_sms, ctx->chunk_kblocks);
+            const int cta_group = ctx->engine == SPECS_ENGINE_TCGEN05_1CTA ? 1
+                                : ctx->engine == SPECS_ENGINE_TCGEN05_2CTA ? 2 : kCtaGroupAuto;
+            const ScorePlan plan = make_score_plan(rows, d, V, ctx->num_sms, ctx->pair_units, cta_group,
+                                                   ctx->chunk_kblocks);
             if (!workspace) return SPECS_ERR_NULL;
             if (workspace_bytes < plan_workspace_bytes(plan)) return SPECS_ERR_WORKSPACE;
             st = launch_score_tcgen05(ctx, plan, hidden, W_vocab, token_ids, static_cast<float*>(workspace), stream);
@@ -349,7 +401,6 @@ int specs_beam_step_host(specs_ctx* ctx, const void* h_hidden, const void* W_voc
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return SPECS_ERR_CUDA;
 
-    const ScorePlan plan = make_score_plan(rows, d, V, ctx->num_sms);
     // carve the arena (every piece 256-byte aligned)
     size_t off = 0;
     auto carve = [&off](size_t bytes) { const size_t at = off; off += (bytes + 255) & ~(size_t)255; return at; };
@@ -358,7 +409,7 @@ int specs_beam_step_host(specs_ctx* ctx, const void* h_hidden, const void* W_voc
     const size_t o_gen = carve((size_t)rows * 4), o_rew = carve((size_t)B * 4), o_uni = carve((size_t)B * 4);
     const size_t o_tok = carve((size_t)rows * 4), o_blk_t = carve((size_t)B * 8), o_blk_g = carve((size_t)B * 8);
     const size_t o_wts = carve((size_t)B * 4), o_cho = carve((size_t)P * 4), o_acc = carve((size_t)P);
-    const size_t ws_bytes = plan_workspace_bytes(plan);
+    const size_t ws_bytes = specs_score_workspace_bytes(ctx, rows, d, V);
     const size_t o_ws = carve(ws_bytes);
     if (off > ctx->arena_bytes) {
         if (ctx->arena) { cudaStreamSynchronize(stream); cudaFree(ctx->arena); ctx->arena = nullptr; ctx->arena_bytes = 0; }

@@ -32,6 +32,7 @@ struct DeviceSetup {
     void* scratch = nullptr;
     uint32_t* status = nullptr;
     int num_sms = 0;
+    int pair_units = 0;
     specs::EncodeTiledFn encode_tiled = nullptr;
 };
 
@@ -62,6 +63,7 @@ int setup_current_device(int device, DeviceSetup* out) {
         s.scratch = scratch;
         s.status = static_cast<uint32_t*>(status);
         s.num_sms = prop.multiProcessorCount;
+        s.pair_units = specs::query_pair_units(device, s.num_sms);   // occupancy query and attributes only
         s.encode_tiled = reinterpret_cast<specs::EncodeTiledFn>(fn);
         s.ready = true;
     }
@@ -89,7 +91,7 @@ extern "C" int specs_score_blocks_noalloc(const void* hidden, const void* W_voca
     int st = setup_current_device(device, &setup);
     if (st != SPECS_OK) return st;
 
-    const specs::ScorePlan plan = specs::make_score_plan(rows, d, V, setup.num_sms);
+    const specs::ScorePlan plan = specs::make_score_plan(rows, d, V, setup.num_sms, setup.pair_units);
     if (specs::plan_workspace_bytes(plan) > (size_t)SPECS_NOALLOC_SCRATCH_BYTES) return SPECS_ERR_LIMIT;
 
     // A context that lives on this stack frame only: it carries what the launchers read
@@ -97,6 +99,7 @@ extern "C" int specs_score_blocks_noalloc(const void* hidden, const void* W_voca
     specs_ctx local;
     local.device = device;
     local.num_sms = setup.num_sms;
+    local.pair_units = setup.pair_units;
     local.encode_tiled = setup.encode_tiled;
     local.d_status = status_word ? status_word : setup.status;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

@@ -6,19 +6,34 @@
 // This is the "computing logits of each token" step of scoring a drafted block with the
 // target model (Section 2 of the paper; Appendix E.3 restricts it to the new block's tokens).
 //
-// One persistent CTA per SM, 384 threads (three warpgroups), three roles:
-//   warp 0      TMA producer: cp.async.bulk.tensor loads of a 128x64 hidden tile and a 256x64
-//               W tile per k-block into a 4-stage, 128-byte-swizzled shared-memory ring.
-//   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32)
-//               into one of two 128-lane x 256-column TMEM buffers.  The reduction over d is
-//               cut into chunks of plan.chunk_kblocks k-blocks; every chunk starts a fresh
-//               accumulator and alternates between the two buffers.
+// Persistent CTAs, one per SM, 384 threads (three warpgroups), three roles:
+//   warp 0      TMA producer: cp.async.bulk.tensor loads of a 128x64 hidden tile and a W tile
+//               per k-block into a ring of 128-byte-swizzled shared-memory stages.
+//   warp 1      MMA issuer: one thread issues tcgen05.mma (N=256, K=16, bf16 -> fp32) into one
+//               of two 128-lane x 256-column TMEM buffers.  The reduction over d is cut into
+//               chunks of plan.chunk_kblocks k-blocks; every chunk starts a fresh accumulator
+//               and alternates between the two buffers.
 //   warps 4-11  epilogue: thread = one row (TMEM lane) x one half (128 columns) of the tile.
 //               After each chunk it adds the chunk's partial logits into fp32 registers
 //               (round-to-nearest), which releases the TMEM buffer for the chunk after next;
 //               after the last chunk it runs, on those registers, the online update of
 //               running max / rescaled sum of 2^x / select of the drafted id's logit.  The
 //               state stays in registers across the CTA's run of vocabulary tiles.
+//
+// Two tile shapes share that body (template parameter kCg = CTAs per work unit):
+//   kCg = 1  one CTA owns a 128-row x 256-column tile: 16 KB of hidden states + 32 KB of W per
+//            k-block, 4 stages.  At 512 tensor clocks per k-block this needs 96 B/clk/SM from
+//            L2, more than the SMs get when all of them stream, so it tops out near 76 % of
+//            the tensor pipe; it remains for problems with a single row tile.
+//   kCg = 2  two CTAs of one cluster own a 256-row x 256-column tile and the leader (cluster
+//            rank 0) issues tcgen05.mma.cta_group::2 over both CTAs' shared memory: each CTA
+//            stages its own 128 hidden rows and only its HALF (128 rows) of the W tile, 32 KB
+//            per k-block (64 B/clk/SM), 6 stages.  Each CTA's TMEM receives its own 128 rows
+//            x 256 columns, so the epilogue is the same.  Barrier traffic across the pair:
+//            the peer's TMA loads complete on the leader's "full" barrier; the leader's
+//            tcgen05.commit arrives on both CTAs' "empty" and "accumulator full" barriers;
+//            both CTAs' epilogue warps arrive on the leader's "accumulator drained" barrier.
+//            W tiles are never multicast: each CTA fetches its own half.
 //
 // Why chunks: the tensor core adds each K=16 group of products into its fp32 accumulator with
 // truncation, so a long reduction carries a bias proportional to the accumulator's magnitude
@@ -35,19 +50,25 @@
 namespace specs {
 namespace {
 
-constexpr int kStages = 4;
 constexpr int kUmmaK = 16;
-constexpr uint32_t kABytes = kBlockM * kBlockK * 2;      // 16 KB
-constexpr uint32_t kBBytes = kBlockN * kBlockK * 2;      // 32 KB
-constexpr uint32_t kStageBytes = kABytes + kBBytes;      // 48 KB
+constexpr int kMaxStages = 8;
+constexpr uint32_t kABytes = kBlockM * kBlockK * 2;      // 16 KB: 128 hidden rows x 64 k
 constexpr int kThreads = 384;                            // three warpgroups: control, epilogue, epilogue
-constexpr int kEpilogueThreads = 256;
+constexpr int kEpilogueWarps = 8;
 constexpr int kHalfN = kBlockN / 2;                      // columns per epilogue thread
 constexpr uint32_t kTmemCols = 512;                      // two 256-column accumulators
-constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kStages * kStageBytes + 256 /*barriers*/;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
 constexpr unsigned long long kDrainLimitNs = 20000000ull;    // 20 ms per stage when draining after an abort
 constexpr float kLog2e = 1.4426950408889634f;
+
+// Per tile shape: W rows staged per CTA and k-block, stage size, ring depth, shared memory.
+template <int kCg> struct Shape {
+    static constexpr int kBRows = kBlockN / kCg;                         // 256, or this CTA's half
+    static constexpr uint32_t kBBytes = kBRows * kBlockK * 2;            // 32 KB / 16 KB
+    static constexpr uint32_t kStageBytes = kABytes + kBBytes;           // 48 KB / 32 KB
+    static constexpr int kStages = kCg == 1 ? 4 : 6;
+    static constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kStages * kStageBytes + 512 /*barriers*/;
+};
 
 // ---- thin PTX wrappers -------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -80,8 +101,37 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false if the CTA-wide abort flag is (or becomes) set.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+// ---- cluster helpers (pair kernel) ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n"
+                 "barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+
+// The abort flag of this CTA and, in the pair kernel, the shared::cluster address of the
+// peer's (0: none): a wait that gives up raises both so that the whole unit winds down.
+struct AbortFlags {
+    volatile uint32_t* own;
+    uint32_t peer;
+};
+// Bounded wait.  Returns false if the abort flag is (or becomes) set.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const AbortFlags& ab,
                                           unsigned long long limit_ns, bool raise) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
@@ -89,9 +139,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 0xFFu) == 0u) {
-            if (raise && *abort_flag) return false;
+            if (raise && *ab.own) return false;
             if (global_timer_ns() - t0 > limit_ns) {
-                if (raise) *abort_flag = 1u;
+                if (raise) {
+                    *ab.own = 1u;
+                    if (ab.peer) st_cluster_u32(ab.peer, 1u);
+                }
                 return false;
             }
         }
@@ -104,6 +157,16 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c_inner), "r"(c_outer), "r"(bar)
         : "memory");
 }
+// The same load issued by a CTA of a pair: the data lands in this CTA's shared memory, the bytes
+// are counted on the barrier at shared::cluster address `cluster_bar` (the leader's).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer,
+                                                 uint32_t cluster_bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c_inner), "r"(c_outer), "r"(cluster_bar)
+        : "memory");
+}
 // 2^x on the special-function unit (relative error about 2^-22; 2^-inf = 0).
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
@@ -114,6 +177,23 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// Commit of the pair's MMAs: arrives on the barrier at this shared-memory offset in BOTH CTAs.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
 }
 __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                             uint32_t accumulate) {
@@ -164,30 +244,39 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16(int m, int n) {
 }
 
 struct SharedLayout {
-    uint64_t full[kStages];      // TMA -> MMA: stage holds data
-    uint64_t empty[kStages];     // MMA -> TMA: stage may be overwritten
+    uint64_t full[kMaxStages];   // TMA -> MMA: stage holds data (pair: only the leader's is used)
+    uint64_t empty[kMaxStages];  // MMA -> TMA: stage may be overwritten
     uint64_t acc_full[2];        // MMA -> epilogue: accumulator complete
-    uint64_t acc_empty[2];       // epilogue -> MMA: accumulator drained
+    uint64_t acc_empty[2];       // epilogue -> MMA: accumulator drained (pair: only the leader's is used)
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
 
-__global__ void __launch_bounds__(kThreads, 1)
-score_tiles_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_w,
-                   const ScorePlan plan, const int32_t* __restrict__ token_ids, float* __restrict__ workspace,
-                   uint32_t* __restrict__ status) {
+template <int kCg>
+__device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, const CUtensorMap& map_w,
+                                                 const ScorePlan& plan, const int32_t* __restrict__ token_ids,
+                                                 float* __restrict__ workspace, uint32_t* __restrict__ status) {
+    using S = Shape<kCg>;
+    constexpr int kStages = S::kStages;
+    constexpr uint32_t kStageBytes = S::kStageBytes;
     extern __shared__ uint8_t smem_raw[];
     // 128-byte-swizzled TMA destinations and UMMA operands must sit on 1024-byte boundaries.
+    // (The dynamic shared-memory window starts at the same offset in both CTAs of a pair, so
+    // the layout below is identical in the two, as the pair's MMA descriptors require.)
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
     uint8_t* tiles = smem_raw + pad;
     SharedLayout* sh = reinterpret_cast<SharedLayout*>(tiles + (size_t)kStages * kStageBytes);
     const uint32_t tiles_addr = smem_u32(tiles);
-    volatile uint32_t* abort_flag = &sh->abort_flag;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int cta = blockIdx.x;
+    const uint32_t rank = (kCg == 2) ? cluster_ctarank() : 0u;   // 0: leader of the pair
+    const int unit = cta / kCg;
+    AbortFlags ab;
+    ab.own = &sh->abort_flag;
+    ab.peer = (kCg == 2) ? mapa_shared(smem_u32(&sh->abort_flag), rank ^ 1u) : 0u;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -196,19 +285,28 @@ score_tiles_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&sh->acc_full[b]), 1);
-            mbar_init(smem_u32(&sh->acc_empty[b]), kEpilogueThreads);
+            mbar_init(smem_u32(&sh->acc_empty[b]), kEpilogueWarps * kCg);   // one arrival per epilogue warp
         }
         sh->abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&sh->tmem_base)), "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        // in the pair kernel warp 1 of BOTH CTAs executes the allocation, with the same arguments
+        if (kCg == 1) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(&sh->tmem_base)), "r"(kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(&sh->tmem_base)), "r"(kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    __syncwarp();
+    if (kCg == 2) cluster_sync_all();     // the peer's barriers are initialised before anything reaches them
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&sh->tmem_base);
 
@@ -220,54 +318,77 @@ score_tiles_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
+            // pair: every load of either CTA is counted on the leader's barrier of the stage
+            const uint32_t full0 = (kCg == 2) ? mapa_shared(smem_u32(&sh->full[0]), 0u) : smem_u32(&sh->full[0]);
             uint32_t stage = 0, phase = 0;
             uint32_t issued = 0;
             bool ok = true;
             for (int w = 0; w < plan.waves && ok; ++w) {
-                int mt, nb, ne;
-                if (!plan_unit(plan, w, cta, &mt, &nb, &ne)) continue;
+                int st, nb, ne;
+                if (!plan_unit(plan, w, unit, &st, &nb, &ne)) continue;
+                const int row0 = (st * kCg + (int)rank) * kBlockM;
                 for (int n = nb; n < ne && ok; ++n) {
+                    const int wrow0 = n * kBlockN + (int)rank * S::kBRows;
                     for (int kb = 0; kb < plan.k_blocks; ++kb) {
-                        if (!mbar_wait(smem_u32(&sh->empty[stage]), phase ^ 1u, abort_flag, kWaitLimitNs, true)) {
+                        if (!mbar_wait(smem_u32(&sh->empty[stage]), phase ^ 1u, ab, kWaitLimitNs, true)) {
                             ok = false;
                             break;
                         }
-                        const uint32_t bar = smem_u32(&sh->full[stage]);
                         const uint32_t a_dst = tiles_addr + stage * kStageBytes;
-                        mbar_arrive_expect_tx(bar, kStageBytes);
-                        tma_load_2d(a_dst, &map_hidden, kb * kBlockK, mt * kBlockM, bar);
-                        tma_load_2d(a_dst + kABytes, &map_w, kb * kBlockK, n * kBlockN, bar);
+                        if (kCg == 1) {
+                            const uint32_t bar = full0 + stage * 8u;
+                            mbar_arrive_expect_tx(bar, kStageBytes);
+                            tma_load_2d(a_dst, &map_hidden, kb * kBlockK, row0, bar);
+                            tma_load_2d(a_dst + kABytes, &map_w, kb * kBlockK, wrow0, bar);
+                        } else {
+                            const uint32_t bar = full0 + stage * 8u;
+                            // the leader expects both CTAs' bytes; the peer's may be counted first
+                            if (rank == 0) mbar_arrive_expect_tx(smem_u32(&sh->full[stage]), 2u * kStageBytes);
+                            tma_load_2d_pair(a_dst, &map_hidden, kb * kBlockK, row0, bar);
+                            tma_load_2d_pair(a_dst + kABytes, &map_w, kb * kBlockK, wrow0, bar);
+                        }
                         ++issued;
                         if (++stage == kStages) { stage = 0; phase ^= 1u; }
                     }
                 }
             }
-            if (!ok) {
+            if (ok) {
+                // Tail: wait until the MMAs that read the last stages have retired, so that no
+                // barrier arrival (in the pair kernel: from the other CTA) is still on its way
+                // to this CTA's shared memory when the CTA exits.
+                for (int i = 0; i < kStages; ++i) {
+                    if (!mbar_wait(smem_u32(&sh->empty[stage]), phase ^ 1u, ab, kWaitLimitNs, true)) break;
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            } else if (kCg == 1 || rank == 0) {
                 // Drain: the last min(issued, kStages) loads may still be landing in shared memory.
                 const uint32_t pending = issued < (uint32_t)kStages ? issued : (uint32_t)kStages;
                 uint32_t s = stage, ph = phase;
                 for (uint32_t i = 0; i < pending; ++i) {
                     if (s == 0) { s = kStages - 1; ph ^= 1u; } else { --s; }
-                    mbar_wait(smem_u32(&sh->full[s]), ph, abort_flag, kDrainLimitNs, false);
+                    mbar_wait(smem_u32(&sh->full[s]), ph, ab, kDrainLimitNs, false);
                 }
+            } else {
+                // The peer cannot poll the leader's barriers: give its own loads in flight a fixed time.
+                const unsigned long long t0 = global_timer_ns();
+                while (global_timer_ns() - t0 < kDrainLimitNs) {}
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = instr_desc_bf16(kBlockM, kBlockN);
+        // ------------------------------------------------------------------ MMA issuer (pair: the leader's)
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = instr_desc_bf16(kBlockM * kCg, kBlockN);
             uint32_t stage = 0, phase = 0;
             uint32_t chunk_count = 0;                        // accumulator hand-overs so far
             bool ok = true;
             for (int w = 0; w < plan.waves && ok; ++w) {
-                int mt, nb, ne;
-                if (!plan_unit(plan, w, cta, &mt, &nb, &ne)) continue;
+                int st, nb, ne;
+                if (!plan_unit(plan, w, unit, &st, &nb, &ne)) continue;
                 for (int n = nb; n < ne && ok; ++n) {
                     for (int kb0 = 0; kb0 < plan.k_blocks && ok; kb0 += plan.chunk_kblocks, ++chunk_count) {
                         const uint32_t buf = chunk_count & 1u;
                         const uint32_t use_phase = (chunk_count >> 1) & 1u;
-                        if (!mbar_wait(smem_u32(&sh->acc_empty[buf]), use_phase ^ 1u, abort_flag, kWaitLimitNs,
-                                       true)) {
+                        if (!mbar_wait(smem_u32(&sh->acc_empty[buf]), use_phase ^ 1u, ab, kWaitLimitNs, true)) {
                             ok = false;
                             break;
                         }
@@ -275,7 +396,7 @@ score_tiles_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_
                         const uint32_t d_tmem = tmem_base + buf * kBlockN;
                         const int kb1 = min(kb0 + plan.chunk_kblocks, plan.k_blocks);
                         for (int kb = kb0; kb < kb1; ++kb) {
-                            if (!mbar_wait(smem_u32(&sh->full[stage]), phase, abort_flag, kWaitLimitNs, true)) {
+                            if (!mbar_wait(smem_u32(&sh->full[stage]), phase, ab, kWaitLimitNs, true)) {
                                 ok = false;
                                 break;
                             }
@@ -287,13 +408,23 @@ score_tiles_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_
                             for (int k = 0; k < kBlockK / kUmmaK; ++k) {
                                 // advancing 16 bf16 (32 bytes) along K inside the swizzled row: +2 in the
                                 // 16-byte units of the descriptor's start-address field
-                                tc_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                            (kb != kb0 || k != 0) ? 1u : 0u);
+                                const uint32_t accumulate = (kb != kb0 || k != 0) ? 1u : 0u;
+                                if (kCg == 1)
+                                    tc_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                                accumulate);
+                                else
+                                    tc_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k),
+                                                     idesc, accumulate);
                             }
-                            tc_commit(smem_u32(&sh->empty[stage]));   // frees the stage once these MMAs retire
+                            // frees the stage (in both CTAs of a pair) once these MMAs retire
+                            if (kCg == 1) tc_commit(smem_u32(&sh->empty[stage]));
+                            else          tc_commit_pair(smem_u32(&sh->empty[stage]));
                             if (++stage == kStages) { stage = 0; phase ^= 1u; }
                         }
-                        if (ok) tc_commit(smem_u32(&sh->acc_full[buf]));  // chunk ready for the epilogue
+                        if (ok) {                            // chunk ready for the epilogue(s)
+                            if (kCg == 1) tc_commit(smem_u32(&sh->acc_full[buf]));
+                            else          tc_commit_pair(smem_u32(&sh->acc_full[buf]));
+                        }
                     }
                 }
             }
@@ -306,12 +437,14 @@ score_tiles_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_
         const int half = (warp - 4) >> 2;                    // which 128 columns of the tile
         const int row_in_tile = quarter * 32 + lane;
         const uint32_t lane_field = static_cast<uint32_t>(quarter * 32) << 16;
+        // "accumulator drained" is counted on the leader's barrier
+        const uint32_t acc_empty0 = (kCg == 2) ? mapa_shared(smem_u32(&sh->acc_empty[0]), 0u) : 0u;
         uint32_t chunk_count = 0;
         bool ok = true;
         for (int w = 0; w < plan.waves && ok; ++w) {
-            int mt, nb, ne;
-            if (!plan_unit(plan, w, cta, &mt, &nb, &ne)) continue;
-            const int64_t row = (int64_t)mt * kBlockM + row_in_tile;
+            int st, nb, ne;
+            if (!plan_unit(plan, w, unit, &st, &nb, &ne)) continue;
+            const int64_t row = (int64_t)(st * kCg + (int)rank) * kBlockM + row_in_tile;
             const int32_t id = (row < plan.rows) ? token_ids[row] : -1;
             // state in base-2 units: run_max = max(z) * log2(e), run_sum = sum 2^(z*log2e - run_max)
             float run_max = -INFINITY, run_sum = 0.0f, picked = -INFINITY;
@@ -320,7 +453,9 @@ score_tiles_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_
                 for (int kb0 = 0; kb0 < plan.k_blocks; kb0 += plan.chunk_kblocks, ++chunk_count) {
                     const uint32_t buf = chunk_count & 1u;
                     const uint32_t use_phase = (chunk_count >> 1) & 1u;
-                    if (!mbar_wait(smem_u32(&sh->acc_full[buf]), use_phase, abort_flag, kWaitLimitNs, true)) {
+                    // the whole warp takes the same decision: __syncwarp below needs every lane
+                    if (!__all_sync(0xffffffffu,
+                                    mbar_wait(smem_u32(&sh->acc_full[buf]), use_phase, ab, kWaitLimitNs, true))) {
                         ok = false;
                         break;
                     }
@@ -343,8 +478,13 @@ score_tiles_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_
                             for (int j = 0; j < 32; ++j) acc[g * 32 + j] += v[j];
                         }
                     }
+                    // the warp's loads are complete: one arrival per warp lets the MMA issuer reuse the buffer
                     tc_fence_before();
-                    mbar_arrive(smem_u32(&sh->acc_empty[buf]));   // the MMA issuer may reuse this buffer
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (kCg == 1) mbar_arrive(smem_u32(&sh->acc_empty[buf]));
+                        else          mbar_arrive_cluster(acc_empty0 + buf * 8u);
+                    }
                 }
                 if (!ok) break;
                 const int col_base = n * kBlockN + half * kHalfN;
@@ -391,11 +531,30 @@ score_tiles_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_
     // ---------------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
+    __syncwarp();
+    if (kCg == 2) cluster_sync_all();     // neither CTA frees TMEM or exits while the other still works
     if (threadIdx.x == 0 && sh->abort_flag != 0u) atomicOr(status, SPECS_DEV_TIMEOUT);
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        if (kCg == 1)
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+score_tiles_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_w,
+                   const ScorePlan plan, const int32_t* __restrict__ token_ids,
+                   float* __restrict__ workspace, uint32_t* __restrict__ status) {
+    score_tiles_body<1>(map_hidden, map_w, plan, token_ids, workspace, status);
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+score_tiles_pair_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_w,
+                        const ScorePlan plan, const int32_t* __restrict__ token_ids,
+                        float* __restrict__ workspace, uint32_t* __restrict__ status) {
+    score_tiles_body<2>(map_hidden, map_w, plan, token_ids, workspace, status);
 }
 
 int encode_bf16_2d(specs_ctx* ctx, CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer,
@@ -413,24 +572,54 @@ int encode_bf16_2d(specs_ctx* ctx, CUtensorMap* map, const void* base, uint64_t 
 
 }  // namespace
 
+int query_pair_units(int device, int num_sms) {
+    // Per device, once: opt both kernels in to their dynamic shared memory (a per-device function
+    // attribute) and ask how many CTA pairs the device keeps resident at once.
+    static int cached[64];
+    static bool done[64] = {};
+    const int slot = device & 63;
+    if (done[slot]) return cached[slot];
+    int units = 0;
+    const bool ok1 = cudaFuncSetAttribute(score_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)Shape<1>::kSmemBytes) == cudaSuccess;
+    const bool ok2 = cudaFuncSetAttribute(score_tiles_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)Shape<2>::kSmemBytes) == cudaSuccess;
+    if (ok2) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(num_sms & ~1), 1, 1);
+        cfg.blockDim = dim3(kThreads, 1, 1);
+        cfg.dynamicSmemBytes = Shape<2>::kSmemBytes;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, score_tiles_pair_kernel, &cfg) == cudaSuccess && clusters > 0)
+            units = clusters < num_sms / 2 ? clusters : num_sms / 2;
+    }
+    cudaGetLastError();                                      // a failed query is not an error of the caller
+    if (!ok1) return 0;                                      // try again on the next call
+    cached[slot] = units;
+    done[slot] = true;
+    return units;
+}
+
 int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan, const void* hidden, const void* w_vocab,
                          const int32_t* token_ids, float* workspace, cudaStream_t stream) {
-    static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+    static_assert(Shape<1>::kSmemBytes <= 227 * 1024 && Shape<2>::kSmemBytes <= 227 * 1024, "shared memory budget");
+    static_assert(Shape<1>::kStages <= kMaxStages && Shape<2>::kStages <= kMaxStages, "barrier arrays");
+    static_assert(sizeof(SharedLayout) <= 512, "barrier block");
+    const bool pair = plan.cta_group == 2;
+    if (pair && (plan.units > ctx->pair_units || (plan.grid & 1))) return SPECS_ERR_CUDA;
+    query_pair_units(ctx->device, ctx->num_sms);             // shared-memory opt-in for this device
     CUtensorMap map_h, map_w;
     int st = encode_bf16_2d(ctx, &map_h, hidden, (uint64_t)plan.d, (uint64_t)plan.rows, kBlockK, kBlockM);
     if (st != SPECS_OK) return st;
-    st = encode_bf16_2d(ctx, &map_w, w_vocab, (uint64_t)plan.d, (uint64_t)plan.V, kBlockK, kBlockN);
+    st = encode_bf16_2d(ctx, &map_w, w_vocab, (uint64_t)plan.d, (uint64_t)plan.V, kBlockK,
+                        pair ? Shape<2>::kBRows : Shape<1>::kBRows);
     if (st != SPECS_OK) return st;
 
-    // The opt-in to more than 48 KB of dynamic shared memory is a per-device function attribute.
-    static bool attr_set[64] = {};
-    const int dev_slot = ctx->device & 63;
-    if (!attr_set[dev_slot]) {
-        cudaError_t e = cudaFuncSetAttribute(score_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)kSmemBytes);
-        if (e != cudaSuccess) return SPECS_ERR_CUDA;
-        attr_set[dev_slot] = true;
-    }
     TimedLaunch* tl = nullptr;
     if (ctx->timing) {
         if (ctx->timed_used == ctx->timed.size()) {
@@ -442,8 +631,12 @@ int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan, const void* hidd
         tl = &ctx->timed[ctx->timed_used++];
         cudaEventRecord(tl->start, stream);
     }
-    score_tiles_kernel<<<plan.grid, kThreads, kSmemBytes, stream>>>(map_h, map_w, plan, token_ids, workspace,
-                                                                    ctx->d_status);
+    if (pair)
+        score_tiles_pair_kernel<<<plan.grid, kThreads, Shape<2>::kSmemBytes, stream>>>(map_h, map_w, plan, token_ids,
+                                                                                      workspace, ctx->d_status);
+    else
+        score_tiles_kernel<<<plan.grid, kThreads, Shape<1>::kSmemBytes, stream>>>(map_h, map_w, plan, token_ids,
+                                                                                 workspace, ctx->d_status);
     if (tl) cudaEventRecord(tl->stop, stream);
     return cuda_status(cudaGetLastError());
 }

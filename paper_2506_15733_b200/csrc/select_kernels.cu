@@ -36,14 +36,17 @@ merge_splits_kernel(const ScorePlan plan, const float* __restrict__ workspace,
     const bool live = row < plan.rows;
     const int64_t row_c = live ? row : plan.rows - 1;
     const int mt = (int)(row_c / kBlockM), r = (int)(row_c % kBlockM);
+    // the row tile's work unit: super tile (cta_group row tiles) and the CTA's rank inside the unit
+    const int cg = plan.cta_group, sup = mt / cg, rank = mt % cg;
     int wave, i, gm, splits;
-    if (mt < plan.full_waves * plan.group_m) {
-        wave = mt / plan.group_m; i = mt % plan.group_m; gm = plan.group_m; splits = plan.split_full;
+    if (sup < plan.full_waves * plan.group_m) {
+        wave = sup / plan.group_m; i = sup % plan.group_m; gm = plan.group_m; splits = plan.split_full;
     } else {
-        wave = plan.full_waves; i = mt - plan.full_waves * plan.group_m; gm = plan.rem_m; splits = plan.split_rem;
+        wave = plan.full_waves; i = sup - plan.full_waves * plan.group_m; gm = plan.rem_m; splits = plan.split_rem;
     }
-    const float* base = workspace + ((size_t)wave * plan.grid + i) * kTripleFloats + r;
-    const size_t stride = (size_t)gm * kTripleFloats;       // next chunk of the same row tile
+    // slot of CTA (unit * cg + rank) with unit = chunk * gm + i
+    const float* base = workspace + ((size_t)wave * plan.grid + (size_t)i * cg + rank) * kTripleFloats + r;
+    const size_t stride = (size_t)gm * cg * kTripleFloats;  // next chunk of the same row tile
     constexpr int kHalf = 3 * kBlockM;                      // second half of the tile's columns
 
     float m = -INFINITY, logit = -INFINITY;

@@ -22,42 +22,55 @@ constexpr int kDefaultChunkKBlocks = 8;      // k-blocks (of 64) per accumulatio
 
 // How the (row tile x vocab tile) grid is cut into persistent work units.
 //
-// Time is cut into waves.  In one wave `gm` consecutive row tiles are live and the vocabulary
-// is cut into `s` contiguous chunks, gm * s <= grid CTAs; CTA c owns row tile (c % gm) of the
-// wave and chunk (c / gm).  CTAs that share a chunk stream the same W tiles at the same pace,
-// so each W tile is fetched from HBM once per wave and hits L2 for the other row tiles, while
-// the wave's hidden-state tiles (gm * 128 * d * 2 bytes) stay L2-resident.  Every wave but the
-// last is "full" (gm = group_m, s = split_full); the last takes the remaining row tiles.
+// A work unit is run by `cta_group` CTAs: one CTA (128 rows), or a pair of CTAs in one
+// cluster (256 rows: the pair issues one tcgen05.mma over both CTAs' shared memory, each CTA
+// stages its own 128 rows of hidden states and only HALF of the 256 W rows of a tile, which
+// cuts the L2 -> shared-memory operand traffic per CTA from 48 KB to 32 KB per k-block).
+// A "super tile" is the cta_group * 128 rows of one unit.
+//
+// Time is cut into waves.  In one wave `gm` consecutive super tiles are live and the
+// vocabulary is cut into `s` contiguous chunks, gm * s <= units; unit u owns super tile
+// (u % gm) of the wave and chunk (u / gm).  Units that share a chunk stream the same W tiles
+// at the same pace, so each W tile is fetched from HBM once per wave and hits L2 for the
+// other super tiles, while the wave's hidden-state tiles stay L2-resident.  Every wave but
+// the last is "full" (gm = group_m, s = split_full); the last takes the remaining super tiles.
 struct ScorePlan {
     int64_t rows;
     int32_t d, V;
     int32_t row_tiles;     // ceil(rows / 128)
     int32_t vocab_tiles;   // ceil(V / 256)
     int32_t k_blocks;      // ceil(d / 64)
-    int32_t grid;          // CTAs launched (= SM count)
-    int32_t group_m;       // row tiles per full wave
+    int32_t cta_group;     // CTAs per work unit: 1, or 2 (cluster pair)
+    int32_t units;         // work units per wave
+    int32_t grid;          // CTAs launched = units * cta_group (also workspace slots per wave)
+    int32_t super_tiles;   // ceil(row_tiles / cta_group)
+    int32_t group_m;       // super tiles per full wave
     int32_t split_full;    // vocab chunks per full wave
     int32_t full_waves;
-    int32_t rem_m;         // row tiles of the last wave (0: none)
+    int32_t rem_m;         // super tiles of the last wave (0: none)
     int32_t split_rem;     // vocab chunks of the last wave
     int32_t waves;         // full_waves + (rem_m > 0)
     int32_t chunk_kblocks; // k-blocks per fresh tensor-core accumulator (chunks are summed in registers)
 };
 
-// Host-side planner (pure arithmetic, no CUDA calls).
-ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms,
-                          int32_t chunk_kblocks = kDefaultChunkKBlocks);
+// cta_group argument of make_score_plan: 0 lets the planner choose between 1 and 2.
+constexpr int kCtaGroupAuto = 0;
+
+// Host-side planner (pure arithmetic, no CUDA calls).  `pair_units` is the number of CTA
+// pairs the device can keep resident (<= num_sms / 2; 0: pairs unavailable).
+ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t pair_units,
+                          int32_t cta_group = kCtaGroupAuto, int32_t chunk_kblocks = kDefaultChunkKBlocks);
 size_t plan_workspace_bytes(const ScorePlan& p);
 
-// Work unit of CTA `cta` in wave `wave`: returns false when the CTA idles in that wave.
-__host__ __device__ inline bool plan_unit(const ScorePlan& p, int wave, int cta,
-                                          int* row_tile, int* n_begin, int* n_end) {
+// Work unit `unit` in wave `wave`: returns false when the unit idles in that wave.
+__host__ __device__ inline bool plan_unit(const ScorePlan& p, int wave, int unit,
+                                          int* super_tile, int* n_begin, int* n_end) {
     int gm, s, base;
     if (wave < p.full_waves) { gm = p.group_m; s = p.split_full; base = wave * p.group_m; }
     else                     { gm = p.rem_m;   s = p.split_rem;  base = p.full_waves * p.group_m; }
-    if (gm <= 0 || cta >= gm * s) return false;
-    const int i = cta % gm, c = cta / gm;
-    *row_tile = base + i;
+    if (gm <= 0 || unit >= gm * s) return false;
+    const int i = unit % gm, c = unit / gm;
+    *super_tile = base + i;
     *n_begin = (int)(((int64_t)c * p.vocab_tiles) / s);
     *n_end   = (int)(((int64_t)(c + 1) * p.vocab_tiles) / s);
     return true;
@@ -76,6 +89,7 @@ struct specs_ctx {
     int device = 0;
     int num_sms = 0;
     int engine = SPECS_ENGINE_TCGEN05;
+    int pair_units = 0;                    // resident CTA pairs of the pair kernel (0: not available)
     int chunk_kblocks = specs::kDefaultChunkKBlocks;   // see specs_set_accum_chunk
     uint32_t* d_status = nullptr;          // device status word (SPECS_DEV_* bits)
     specs::EncodeTiledFn encode_tiled = nullptr;
@@ -91,6 +105,9 @@ struct specs_ctx {
 namespace specs {
 
 // ---- kernel launchers (each enqueues on `stream`, returns a specs_status) ---------------------
+// CTA pairs of the pair kernel that the current device keeps resident at once (cached per
+// device; also opts both kernels in to their dynamic shared memory).  0 if pairs cannot launch.
+int query_pair_units(int device, int num_sms);
 int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan, const void* hidden, const void* w_vocab,
                          const int32_t* token_ids, float* workspace, cudaStream_t stream);
 int launch_score_simt(specs_ctx* ctx, const void* hidden, const void* w_vocab, const int32_t* token_ids,

@@ -60,11 +60,17 @@ def check_selection_logic(x, got, beta, tau, gen_blk):
     return int(sure.sum())
 
 
-def test_step7b_all_rows_all_betas(ctx):
+@pytest.mark.parametrize("engine", [binding.ENGINE_TCGEN05, binding.ENGINE_TCGEN05_1CTA])
+def test_step7b_all_rows_all_betas(ctx, engine):
+    # default engine (CTA pairs at this size) and the single-CTA tile shape
     cfg = I.CONFIGS["step7b"]
     x = I.make_step_inputs(cfg)
     s = DeviceStep(ctx, x)
-    got = s.step(cfg.betas[0], 0.7)
+    ctx.set_engine(engine)
+    try:
+        got = s.step(cfg.betas[0], 0.7)
+    finally:
+        ctx.set_engine(binding.ENGINE_TCGEN05)
     w64 = O.bf16_bits_to_f64(x.w_vocab)
     all_rows = np.arange(x.rows)
     want_tok, err = check_sampled_rows(x, got["tok_logprob"], all_rows, w64)

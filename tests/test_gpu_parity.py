@@ -33,7 +33,10 @@ def small_config(name, rows_per_block, problems, beams, d, V, seed, **kw):
 
 # ------------------------------------------------------------------------------- tiny, both engines
 
-@pytest.mark.parametrize("engine", [binding.ENGINE_SIMT, binding.ENGINE_TCGEN05])
+TC_ENGINES = [binding.ENGINE_TCGEN05_1CTA, binding.ENGINE_TCGEN05_2CTA]   # both tile shapes of the tensor-core kernel
+
+
+@pytest.mark.parametrize("engine", [binding.ENGINE_SIMT, binding.ENGINE_TCGEN05] + TC_ENGINES)
 def test_tiny_config_full_step(ctx, engine):
     x = I.make_step_inputs(I.CONFIGS["tiny"])
     ctx.set_engine(engine)
@@ -59,14 +62,20 @@ EDGE_CASES = [
     ((3, 40), 3, 5, 256, 2500),      # ragged blocks, several tiles, vocab tail of 196
     ((16, 16), 2, 4, 520, 257),      # vocab tile with a single valid column in its last tile
     ((50, 50), 1, 6, 1024, 4096),    # exact multiples everywhere
+    ((75, 75), 1, 4, 128, 700),      # three row tiles: the last CTA pair has one CTA without rows
 ]
 
 
+@pytest.mark.parametrize("engine", TC_ENGINES)
 @pytest.mark.parametrize("blk,P,n,d,V", EDGE_CASES)
-def test_edge_shapes(ctx, blk, P, n, d, V):
+def test_edge_shapes(ctx, blk, P, n, d, V, engine):
     cfg = small_config("edge", blk, P, n, d, V, seed=4000 + d + V)
     x = I.make_step_inputs(cfg)
-    got = DeviceStep(ctx, x).step(1.0, 0.5)
+    ctx.set_engine(engine)
+    try:
+        got = DeviceStep(ctx, x).step(1.0, 0.5)
+    finally:
+        ctx.set_engine(binding.ENGINE_TCGEN05)
     want = oracle_step(x, 1.0, 0.5)
     assert_step_matches(got, want, x.cand_offsets, x.block_offsets)
     assert ctx.device_status() == 0
@@ -105,16 +114,21 @@ def test_zero_rows_is_a_noop(ctx):
 
 # ------------------------------------------------------------------------------- several waves of work units
 
+@pytest.mark.parametrize("engine", TC_ENGINES)
 @pytest.mark.parametrize("rows_total,d,V", [(20000, 64, 1000), (10000, 1536, 2048), (40000, 128, 520)])
-def test_multi_wave_plans(ctx, rows_total, d, V):
+def test_multi_wave_plans(ctx, rows_total, d, V, engine):
     sms = ctx.sm_count()
-    plan = binding.score_plan(rows_total, d, V, sms)
+    plan = binding.score_plan(rows_total, d, V, sms, 1 if engine == binding.ENGINE_TCGEN05_1CTA else 2)
     assert plan["waves"] >= 2, plan
     blocks = 40
     cfg = small_config("waves", (rows_total // blocks, rows_total // blocks), 4, blocks // 4, d, V,
                        seed=4200 + d, w_sigma=0.5 / math.sqrt(d) * 4)
     x = I.make_step_inputs(cfg)
-    got = DeviceStep(ctx, x).step(1.0, 0.6)
+    ctx.set_engine(engine)
+    try:
+        got = DeviceStep(ctx, x).step(1.0, 0.6)
+    finally:
+        ctx.set_engine(binding.ENGINE_TCGEN05)
     want = oracle_step(x, 1.0, 0.6)
     assert_step_matches(got, want, x.cand_offsets, x.block_offsets)
     assert ctx.device_status() == 0
@@ -128,7 +142,7 @@ def test_out_of_range_token_is_nan_and_flagged(ctx):
     x.token_ids = x.token_ids.copy()
     x.token_ids[3] = 300
     x.token_ids[9] = -2
-    for engine in (binding.ENGINE_TCGEN05, binding.ENGINE_SIMT):
+    for engine in (binding.ENGINE_TCGEN05_1CTA, binding.ENGINE_TCGEN05_2CTA, binding.ENGINE_SIMT):
         ctx.set_engine(engine)
         try:
             s = DeviceStep(ctx, x)

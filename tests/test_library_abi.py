@@ -39,11 +39,12 @@ def test_status_strings(lib):
 
 
 def test_host_validation_without_a_device(lib):
-    out = (ctypes.c_int32 * 12)()
-    assert lib.specs_score_plan(128, 12, 100, 148, out) == 2        # d % 8 != 0
-    assert lib.specs_score_plan(-1, 16, 100, 148, out) == 2
-    assert lib.specs_score_plan(128, 16, 0, 148, out) == 2
-    assert lib.specs_score_plan(128, 16, 100, 148, None) == 1
+    out = (ctypes.c_int32 * 16)()
+    assert lib.specs_score_plan(128, 12, 100, 148, 0, out) == 2     # d % 8 != 0
+    assert lib.specs_score_plan(-1, 16, 100, 148, 0, out) == 2
+    assert lib.specs_score_plan(128, 16, 0, 148, 0, out) == 2
+    assert lib.specs_score_plan(128, 16, 100, 148, 3, out) == 2     # no such tile shape
+    assert lib.specs_score_plan(128, 16, 100, 148, 0, None) == 1
     # calls that need a context refuse a NULL one instead of crashing
     assert lib.specs_destroy(None) == 0
     assert lib.specs_set_engine(None, 0) == 1
@@ -59,39 +60,56 @@ PLAN_CASES = [
 ]
 
 
+@pytest.mark.parametrize("cta_group", [0, 1, 2])
 @pytest.mark.parametrize("rows,d,V,sms", PLAN_CASES)
-def test_plan_covers_every_tile_exactly_once(lib, rows, d, V, sms):
-    p = binding.score_plan(rows, d, V, sms)
+def test_plan_covers_every_tile_exactly_once(lib, rows, d, V, sms, cta_group):
+    p = binding.score_plan(rows, d, V, sms, cta_group)
+    cg = p["cta_group"]
+    assert cg in (1, 2) and (cta_group == 0 or cg == cta_group)
     assert p["row_tiles"] == -(-rows // 128) and p["vocab_tiles"] == -(-V // 256) and p["k_blocks"] == -(-d // 64)
-    assert p["grid"] == sms and p["waves"] == p["full_waves"] + (1 if p["rem_m"] else 0)
-    assert p["group_m"] * p["split_full"] <= sms
-    assert p["full_waves"] * p["group_m"] + p["rem_m"] == p["row_tiles"]
+    assert p["super_tiles"] == -(-p["row_tiles"] // cg)
+    assert p["units"] == sms // cg and p["grid"] == p["units"] * cg
+    assert p["waves"] == p["full_waves"] + (1 if p["rem_m"] else 0)
+    assert p["group_m"] * p["split_full"] <= p["units"]
+    assert p["full_waves"] * p["group_m"] + p["rem_m"] == p["super_tiles"]
     if p["rem_m"]:
-        assert 1 <= p["split_rem"] and p["rem_m"] * p["split_rem"] <= sms
-    assert p["workspace_bytes"] == p["waves"] * sms * 2 * 3 * 128 * 4
-    assert p["workspace_bytes"] < 128 * rows + (1 << 20)              # never anything like rows x V
+        assert 1 <= p["split_rem"] and p["rem_m"] * p["split_rem"] <= p["units"]
+    assert p["workspace_bytes"] == p["waves"] * p["grid"] * 2 * 3 * 128 * 4
+    assert p["workspace_bytes"] < 256 * rows + (1 << 20)              # never anything like rows x V
     covered = {}
-    busiest = 0
     for w in range(p["waves"]):
-        for c in range(sms):
-            mt, nb, ne = binding.score_plan_unit(rows, d, V, sms, w, c)
+        for c in range(p["grid"]):
+            mt, nb, ne = binding.score_plan_unit(rows, d, V, sms, w, c, cta_group)
             if mt < 0:
                 continue
             assert 0 <= mt < p["row_tiles"] and 0 <= nb < ne <= p["vocab_tiles"]
+            if cg == 2:
+                # both CTAs of a pair work on the same vocabulary tiles, on adjacent row tiles
+                mt2, nb2, ne2 = binding.score_plan_unit(rows, d, V, sms, w, c ^ 1, cta_group)
+                assert mt2 in (-1, mt ^ 1) and (mt2 < 0 or (nb2, ne2) == (nb, ne))
             for n in range(nb, ne):
                 assert (mt, n) not in covered
                 covered[(mt, n)] = (w, c)
-            busiest = max(busiest, ne - nb)
+        assert binding.score_plan_unit(rows, d, V, sms, w, p["grid"], cta_group)[0] == -1
     assert len(covered) == p["row_tiles"] * p["vocab_tiles"]
 
 
 def test_plan_balance_on_the_benchmark_shapes(lib):
-    # makespan in tiles per CTA versus the ideal total / grid
-    for rows, d, V in [(1024, 3584, 151936), (65536, 3584, 151936), (131072, 5120, 152064), (65536, 1536, 151936)]:
-        p = binding.score_plan(rows, d, V, 148)
-        span = 0
-        for w in range(p["waves"]):
-            span += max(ne - nb for mt, nb, ne in
-                        (binding.score_plan_unit(rows, d, V, 148, w, c) for c in range(148)) if mt >= 0)
-        ideal = p["row_tiles"] * p["vocab_tiles"] / 148
-        assert span <= 1.06 * ideal + 1, (rows, d, V, span, ideal, p)
+    # makespan in tiles per unit versus the ideal total / units, for both tile shapes
+    for rows, d, V in [(1024, 3584, 151936), (65536, 3584, 151936), (131072, 5120, 152064), (65536, 1536, 151936),
+                       (20893, 3584, 151936)]:
+        for cg in (1, 2):
+            p = binding.score_plan(rows, d, V, 148, cg)
+            span = 0
+            for w in range(p["waves"]):
+                span += max(ne - nb for mt, nb, ne in
+                            (binding.score_plan_unit(rows, d, V, 148, w, c, cg) for c in range(p["grid"])) if mt >= 0)
+            ideal = p["super_tiles"] * p["vocab_tiles"] / p["units"]
+            assert span <= 1.06 * ideal + 1, (rows, d, V, cg, span, ideal, p)
+
+
+def test_planner_prefers_pairs_except_for_a_single_row_tile(lib):
+    assert binding.score_plan(1024, 3584, 151936, 148)["cta_group"] == 2
+    assert binding.score_plan(65536, 3584, 151936, 148)["cta_group"] == 2
+    assert binding.score_plan(100, 3584, 151936, 148)["cta_group"] == 1     # 256-row tiles would be half empty
+    assert binding.score_plan(1024, 3584, 151936, 1)["cta_group"] == 1      # no pair fits on one SM
