@@ -53,6 +53,7 @@ typedef enum specs_status {
 /* Bits of the device status word returned by specs_device_status(). */
 #define SPECS_DEV_TIMEOUT      0x1u
 #define SPECS_DEV_TOKEN_RANGE  0x2u
+#define SPECS_DEV_ACCUM_RANGE  0x4u   /* advisory, see specs_set_accum_chunk; does not change a return value */
 
 /* Scoring engines (see specs_set_engine). */
 #define SPECS_ENGINE_TCGEN05      0   /* tensor-core path: TMA + tcgen05.mma + TMEM, fused epilogue (default);
@@ -76,12 +77,26 @@ int specs_destroy(specs_ctx* ctx);
  * for and the device cannot launch them). */
 int specs_set_engine(specs_ctx* ctx, int engine);
 
-/* Length, in elements of d, of one tensor-core accumulation chunk (a multiple of
- * 64; default 512; 0 = accumulate the whole of d in one go).  The tensor core adds
- * into its fp32 accumulator with truncation, which biases long reductions of large
- * logits (about -5e-3 at |logit| = 700, d = 5120); the kernel therefore restarts the
- * accumulator every chunk and sums the chunks in registers with round-to-nearest,
- * which divides the bias by the number of chunks.  Shorter chunks cost epilogue time. */
+/* How the tensor-core kernel cuts the reduction over d into accumulation chunks.
+ * The tensor core adds every K = 16 group of products into its fp32 accumulator
+ * with truncation, which biases long reductions of large logits (about -5e-3 at
+ * |logit| = 700, d = 5120).  The kernel therefore restarts the accumulator every
+ * chunk and sums the chunks in registers with round-to-nearest, which divides the
+ * bias by the number of chunks; every restart costs a read of the accumulator out
+ * of tensor memory (about 2 % of a tile's time each at d = 3584).
+ *   k_elements > 0 (a multiple of 64): fixed chunks of that length.
+ *   k_elements = 0: one accumulator over the whole of d.
+ *   SPECS_ACCUM_ADAPTIVE (default): 512-element chunks for the first two vocabulary
+ *     tiles of each run of tiles a CTA (pair) scores for its rows; the largest
+ *     |logit| of the first tile then sets the chunk length of the remaining tiles:
+ *     as many K = 16 accumulations as keep (count x fp32 spacing at twice that
+ *     magnitude) below 2.5e-4, never shorter than 512 elements.  Logits of a few
+ *     units (the usual LM-head range) run unchunked, logits in the hundreds keep the
+ *     512-element chunks.  If a later tile of the run holds a positive logit, or the
+ *     drafted id's logit, beyond the binade assumed, the results stand but the
+ *     advisory bit SPECS_DEV_ACCUM_RANGE is set: those rows may carry a few 1e-3 of
+ *     accumulation bias; rescore with a fixed chunk if that matters. */
+#define SPECS_ACCUM_ADAPTIVE (-1)
 int specs_set_accum_chunk(specs_ctx* ctx, int32_t k_elements);
 
 /* Number of SMs the context schedules over (the persistent grid is one CTA per SM,

@@ -24,6 +24,8 @@ ENGINE_TCGEN05_1CTA = 2
 ENGINE_TCGEN05_2CTA = 3
 DEV_TIMEOUT = 0x1
 DEV_TOKEN_RANGE = 0x2
+DEV_ACCUM_RANGE = 0x4
+ACCUM_ADAPTIVE = -1
 
 _vp, _i32, _i64, _f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
 

@@ -62,7 +62,7 @@ double fill_plan(ScorePlan* p, int32_t cta_group, int32_t units) {
 }  // namespace
 
 ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t pair_units,
-                          int32_t cta_group, int32_t chunk_kblocks) {
+                          int32_t cta_group, int32_t chunk_kblocks, bool adaptive) {
     ScorePlan p;
     std::memset(&p, 0, sizeof(p));
     p.rows = rows; p.d = d; p.V = V;
@@ -70,6 +70,7 @@ ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, i
     p.vocab_tiles = (V + kBlockN - 1) / kBlockN;
     p.k_blocks = (d + kBlockK - 1) / kBlockK;
     p.chunk_kblocks = (chunk_kblocks > 0 && chunk_kblocks < p.k_blocks) ? chunk_kblocks : p.k_blocks;
+    p.adaptive = (adaptive && p.chunk_kblocks < p.k_blocks) ? 1 : 0;
     if (pair_units <= 0 && cta_group == 2) cta_group = 1;      // pairs unavailable on this device
     if (cta_group == 1 || pair_units <= 0) {
         fill_plan(&p, 1, num_sms);
@@ -208,8 +209,14 @@ int specs_set_engine(specs_ctx* ctx, int engine) {
 
 int specs_set_accum_chunk(specs_ctx* ctx, int32_t k_elements) {
     if (!ctx) return SPECS_ERR_NULL;
+    if (k_elements == SPECS_ACCUM_ADAPTIVE) {
+        ctx->chunk_kblocks = kDefaultChunkKBlocks;
+        ctx->accum_adaptive = true;
+        return SPECS_OK;
+    }
     if (k_elements < 0 || (k_elements % kBlockK) != 0) return SPECS_ERR_SHAPE;
     ctx->chunk_kblocks = k_elements / kBlockK;               // 0: one accumulator over the whole of d
+    ctx->accum_adaptive = false;
     return SPECS_OK;
 }
 
@@ -276,7 +283,7 @@ int specs_score_blocks(specs_ctx* ctx, const void* hidden, const void* W_vocab, 
             const int cta_group = ctx->engine == SPECS_ENGINE_TCGEN05_1CTA ? 1
                                 : ctx->engine == SPECS_ENGINE_TCGEN05_2CTA ? 2 : kCtaGroupAuto;
             const ScorePlan plan = make_score_plan(rows, d, V, ctx->num_sms, ctx->pair_units, cta_group,
-                                                   ctx->chunk_kblocks);
+                                                   ctx->chunk_kblocks, ctx->accum_adaptive);
             if (!workspace) return SPECS_ERR_NULL;
             if (workspace_bytes < plan_workspace_bytes(plan)) return SPECS_ERR_WORKSPACE;
             st = launch_score_tcgen05(ctx, plan, hidden, W_vocab, token_ids, static_cast<float*>(workspace), stream);

@@ -39,7 +39,13 @@
 // truncation, so a long reduction carries a bias proportional to the accumulator's magnitude
 // times the number of accumulations (about -5e-3 on logits near 700 at d = 5120).  Restarting
 // the accumulator every 512 elements and summing the chunks in registers with round-to-nearest
-// divides that bias by the number of chunks.
+// divides that bias by the number of chunks.  Each restart costs a read of the accumulator out
+// of TMEM, which holds up the tensor pipe for about 500 clocks, so chunks are only as short as
+// the logits demand: with plan.adaptive the first two vocabulary tiles of a run use the base
+// chunk; the epilogue warps publish the largest |logit| of the first tile, and from the third
+// tile on the MMA issuer and the epilogue both derive the chunk length from it
+// (adaptive_chunk_kblocks).  The hand-over is a barrier ("mode") on which every epilogue warp of
+// the unit arrives after writing its maximum into every CTA of the unit.
 // Every mbarrier wait is bounded; on expiry the CTA raises SPECS_DEV_TIMEOUT, all roles leave
 // their loops, the producer waits (bounded) for its copies in flight, TMEM is freed and the
 // kernel returns.
@@ -54,6 +60,14 @@ constexpr int kUmmaK = 16;
 constexpr int kMaxStages = 8;
 constexpr uint32_t kABytes = kBlockM * kBlockK * 2;      // 16 KB: 128 hidden rows x 64 k
 constexpr int kThreads = 384;                            // three warpgroups: control, epilogue, epilogue
+// Registers per thread after the warpgroups re-balance them (setmaxnreg).  The increase waits,
+// without bound, until the CTA's own allocation (launch registers x threads) has that much to
+// give, so the two budgets must fit into it.
+constexpr int kLaunchRegs = 168;                         // what __launch_bounds__(384, 1) yields
+constexpr int kControlRegs = 120;
+constexpr int kEpilogueRegs = 184;
+static_assert(128 * kControlRegs + 256 * kEpilogueRegs <= kThreads * kLaunchRegs,
+              "setmaxnreg budgets exceed the CTA's register allocation: the increase would never return");
 constexpr int kEpilogueWarps = 8;
 constexpr int kHalfN = kBlockN / 2;                      // columns per epilogue thread
 constexpr uint32_t kTmemCols = 512;                      // two 256-column accumulators
@@ -124,6 +138,24 @@ __device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v
     asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
 }
 
+// try_wait whose acquire covers writes made by the other CTA of the pair before its arrival
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t cluster_addr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v) : "memory");
+}
+
 // The abort flag of this CTA and, in the pair kernel, the shared::cluster address of the
 // peer's (0: none): a wait that gives up raises both so that the whole unit winds down.
 struct AbortFlags {
@@ -132,12 +164,12 @@ struct AbortFlags {
 };
 // Bounded wait.  Returns false if the abort flag is (or becomes) set.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const AbortFlags& ab,
-                                          unsigned long long limit_ns, bool raise) {
-    if (mbar_try_wait(bar, parity)) return true;
+                                          unsigned long long limit_ns, bool raise, bool cluster_acquire = false) {
+    if (cluster_acquire ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     uint32_t spins = 0;
     for (;;) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (cluster_acquire ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
         if ((++spins & 0xFFu) == 0u) {
             if (raise && *ab.own) return false;
             if (global_timer_ns() - t0 > limit_ns) {
@@ -226,6 +258,16 @@ __device__ __forceinline__ void tmem_ld_32cols(uint32_t taddr, float (&v)[32]) {
     for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
 }
 
+// The same for 16 consecutive columns, straight into float registers.
+__device__ __forceinline__ void tmem_ld_16cols(uint32_t taddr, float (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
+        "tcgen05.wait::ld.sync.aligned;\n"
+        : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]), "=f"(v[8]), "=f"(v[9]), "=f"(v[10]), "=f"(v[11]), "=f"(v[12]), "=f"(v[13]), "=f"(v[14]), "=f"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+
 // Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (64
 // elements) long, written by TMA with the 128-byte swizzle: 8-row groups are 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t saddr) {
@@ -248,9 +290,39 @@ struct SharedLayout {
     uint64_t empty[kMaxStages];  // MMA -> TMA: stage may be overwritten
     uint64_t acc_full[2];        // MMA -> epilogue: accumulator complete
     uint64_t acc_empty[2];       // epilogue -> MMA: accumulator drained (pair: only the leader's is used)
+    uint64_t mode;               // epilogue warps -> MMA issuer and epilogue: |logit| maxima published
+    float absmax[2 * kEpilogueWarps];   // largest |logit| of the run's first tile, per epilogue warp of the unit
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
+
+// Chunk length (in k-blocks of 64) for logits whose magnitude stays below twice `absmax`.
+// One accumulation (K = 16) truncates the fp32 accumulator toward zero by at most one spacing of
+// its magnitude.  The chunk gets as many accumulations as keep (count x spacing) under 2.5e-4,
+// an eighth of the 2e-3 tolerance on a token log-probability; it is never shorter than `base`.
+// `*bound` receives the magnitude up to which that spacing holds (the top of the binade).
+__device__ __forceinline__ int adaptive_chunk_kblocks(float absmax, int base, int k_blocks, float* bound) {
+    *bound = INFINITY;                                       // no claim when the base chunk is kept
+    const float a = fmaxf(2.0f * absmax, 1.0f);
+    if (!(a < 128.0f)) return base;                          // also NaN and inf
+    const int e = ((__float_as_int(a) >> 23) & 0xff) - 126;  // a = m * 2^e with m in [0.5, 1)
+    const float n_acc = ldexpf(2.5e-4f, 24 - e);             // spacing of [2^(e-1), 2^e) is 2^(e-24)
+    int kb = (int)(n_acc * 0.25f);                           // four accumulations per k-block
+    if (kb <= base) return base;
+    *bound = ldexpf(1.0f, e);
+    if (kb >= k_blocks) return k_blocks;
+    const int chunks = (k_blocks + kb - 1) / kb;             // equal chunks
+    return (k_blocks + chunks - 1) / chunks;
+}
+// Largest published maximum of the unit (8 values per CTA of the unit).
+template <int kCg>
+__device__ __forceinline__ float read_absmax(const SharedLayout* sh) {
+    const volatile float* p = sh->absmax;
+    float m = 0.0f;
+#pragma unroll
+    for (int i = 0; i < kEpilogueWarps * kCg; ++i) m = fmaxf(m, p[i]);
+    return m;
+}
 
 template <int kCg>
 __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, const CUtensorMap& map_w,
@@ -287,6 +359,7 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
             mbar_init(smem_u32(&sh->acc_full[b]), 1);
             mbar_init(smem_u32(&sh->acc_empty[b]), kEpilogueWarps * kCg);   // one arrival per epilogue warp
         }
+        mbar_init(smem_u32(&sh->mode), kEpilogueWarps * kCg);
         sh->abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -311,10 +384,10 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&sh->tmem_base);
 
     // Registers move from the control warpgroup (which needs few) to the two epilogue warpgroups
-    // (128 fp32 partial logits per thread): 128*120 + 256*184 <= 64K.  Each setmaxnreg sits at the
+    // (128 fp32 partial logits per thread).  Each setmaxnreg sits at the
     // top of the code it governs so that the register allocator sees which budget applies where.
     if (warp < 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 120;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kControlRegs));
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -380,12 +453,24 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
             constexpr uint32_t idesc = instr_desc_bf16(kBlockM * kCg, kBlockN);
             uint32_t stage = 0, phase = 0;
             uint32_t chunk_count = 0;                        // accumulator hand-overs so far
+            uint32_t mode_runs = 0;                          // completed phases of the "mode" barrier
             bool ok = true;
             for (int w = 0; w < plan.waves && ok; ++w) {
                 int st, nb, ne;
                 if (!plan_unit(plan, w, unit, &st, &nb, &ne)) continue;
+                const bool adapt_run = plan.adaptive && (ne - nb) >= 3;
+                int ck = plan.chunk_kblocks;                 // k-blocks per chunk of the current tile
                 for (int n = nb; n < ne && ok; ++n) {
-                    for (int kb0 = 0; kb0 < plan.k_blocks && ok; kb0 += plan.chunk_kblocks, ++chunk_count) {
+                    if (adapt_run && n == nb + 2) {
+                        if (!mbar_wait(smem_u32(&sh->mode), mode_runs & 1u, ab, kWaitLimitNs, true, true)) {
+                            ok = false;
+                            break;
+                        }
+                        ++mode_runs;
+                        float bound;
+                        ck = adaptive_chunk_kblocks(read_absmax<kCg>(sh), plan.chunk_kblocks, plan.k_blocks, &bound);
+                    }
+                    for (int kb0 = 0; kb0 < plan.k_blocks && ok; kb0 += ck, ++chunk_count) {
                         const uint32_t buf = chunk_count & 1u;
                         const uint32_t use_phase = (chunk_count >> 1) & 1u;
                         if (!mbar_wait(smem_u32(&sh->acc_empty[buf]), use_phase ^ 1u, ab, kWaitLimitNs, true)) {
@@ -394,7 +479,7 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                         }
                         tc_fence_after();
                         const uint32_t d_tmem = tmem_base + buf * kBlockN;
-                        const int kb1 = min(kb0 + plan.chunk_kblocks, plan.k_blocks);
+                        const int kb1 = min(kb0 + ck, plan.k_blocks);
                         for (int kb = kb0; kb < kb1; ++kb) {
                             if (!mbar_wait(smem_u32(&sh->full[stage]), phase, ab, kWaitLimitNs, true)) {
                                 ok = false;
@@ -431,7 +516,7 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
         }
     }
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 184;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kEpilogueRegs));
         // ------------------------------------------------------------------ epilogue (warps 4..11)
         const int quarter = warp & 3;                        // TMEM lanes 32*quarter .. +31 belong to this warp
         const int half = (warp - 4) >> 2;                    // which 128 columns of the tile
@@ -440,17 +525,30 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
         // "accumulator drained" is counted on the leader's barrier
         const uint32_t acc_empty0 = (kCg == 2) ? mapa_shared(smem_u32(&sh->acc_empty[0]), 0u) : 0u;
         uint32_t chunk_count = 0;
+        uint32_t mode_runs = 0;
         bool ok = true;
         for (int w = 0; w < plan.waves && ok; ++w) {
             int st, nb, ne;
             if (!plan_unit(plan, w, unit, &st, &nb, &ne)) continue;
+            const bool adapt_run = plan.adaptive && (ne - nb) >= 3;
+            int ck = plan.chunk_kblocks;                     // k-blocks per chunk of the current tile
+            float assumed = INFINITY;                        // magnitude the lengthened chunks were sized for
             const int64_t row = (int64_t)(st * kCg + (int)rank) * kBlockM + row_in_tile;
             const int32_t id = (row < plan.rows) ? token_ids[row] : -1;
             // state in base-2 units: run_max = max(z) * log2(e), run_sum = sum 2^(z*log2e - run_max)
             float run_max = -INFINITY, run_sum = 0.0f, picked = -INFINITY;
             for (int n = nb; n < ne && ok; ++n) {
+                if (adapt_run && n == nb + 2) {
+                    if (!__all_sync(0xffffffffu,
+                                    mbar_wait(smem_u32(&sh->mode), mode_runs & 1u, ab, kWaitLimitNs, true, true))) {
+                        ok = false;
+                        break;
+                    }
+                    ++mode_runs;
+                    ck = adaptive_chunk_kblocks(read_absmax<kCg>(sh), plan.chunk_kblocks, plan.k_blocks, &assumed);
+                }
                 float acc[kHalfN];                           // this thread's 128 logits of the tile
-                for (int kb0 = 0; kb0 < plan.k_blocks; kb0 += plan.chunk_kblocks, ++chunk_count) {
+                for (int kb0 = 0; kb0 < plan.k_blocks; kb0 += ck, ++chunk_count) {
                     const uint32_t buf = chunk_count & 1u;
                     const uint32_t use_phase = (chunk_count >> 1) & 1u;
                     // the whole warp takes the same decision: __syncwarp below needs every lane
@@ -470,12 +568,13 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                             for (int j = 0; j < 32; ++j) acc[g * 32 + j] = v[j];
                         }
                     } else {
+                        // 16 columns at a time: with 128 running sums live, a 32-register landing area spills
 #pragma unroll
-                        for (int g = 0; g < kHalfN / 32; ++g) {
-                            float v[32];
-                            tmem_ld_32cols(taddr + g * 32, v);
+                        for (int g = 0; g < kHalfN / 16; ++g) {
+                            float v[16];
+                            tmem_ld_16cols(taddr + g * 16, v);
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) acc[g * 32 + j] += v[j];
+                            for (int j = 0; j < 16; ++j) acc[g * 16 + j] += v[j];
                         }
                     }
                     // the warp's loads are complete: one arrival per warp lets the MMA issuer reuse the buffer
@@ -488,6 +587,28 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                 }
                 if (!ok) break;
                 const int col_base = n * kBlockN + half * kHalfN;
+                if (adapt_run && n == nb) {
+                    // first tile of the run: publish this warp's largest |logit| to every CTA of the unit
+                    float amax = 0.0f;
+#pragma unroll
+                    for (int j = 0; j < kHalfN; ++j)
+                        amax = (col_base + j < plan.V) ? fmaxf(amax, fabsf(acc[j])) : amax;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+                    if (lane == 0) {
+                        const int slot = (int)rank * kEpilogueWarps + (warp - 4);
+                        if (kCg == 1) {
+                            sh->absmax[slot] = amax;
+                            mbar_arrive(smem_u32(&sh->mode));
+                        } else {
+#pragma unroll
+                            for (uint32_t r = 0; r < 2; ++r) {
+                                st_cluster_f32(mapa_shared(smem_u32(&sh->absmax[slot]), r), amax);
+                                mbar_arrive_cluster(mapa_shared(smem_u32(&sh->mode), r));
+                            }
+                        }
+                    }
+                }
 #pragma unroll
                 for (int g = 0; g < kHalfN / 32; ++g) {
                     const int col0 = col_base + g * 32;
@@ -520,6 +641,9 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                 }
             }
             if (ok) {
+                // a positive logit or the drafted id's logit beyond the magnitude the chunks were sized for
+                if (run_max > assumed * kLog2e || (picked != -INFINITY && fabsf(picked) > assumed))
+                    atomicOr(status, SPECS_DEV_ACCUM_RANGE);
                 float* slot = workspace + ((size_t)w * plan.grid + cta) * kTripleFloats + half * 3 * kBlockM;
                 slot[row_in_tile] = run_max;
                 slot[kBlockM + row_in_tile] = run_sum;

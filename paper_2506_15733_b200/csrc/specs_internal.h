@@ -51,6 +51,8 @@ struct ScorePlan {
     int32_t split_rem;     // vocab chunks of the last wave
     int32_t waves;         // full_waves + (rem_m > 0)
     int32_t chunk_kblocks; // k-blocks per fresh tensor-core accumulator (chunks are summed in registers)
+    int32_t adaptive;      // 1: from the third vocabulary tile of a run on, lengthen the chunks as far as the
+                           //    logit magnitude seen in the run's first tile allows (see score_tcgen05.cu)
 };
 
 // cta_group argument of make_score_plan: 0 lets the planner choose between 1 and 2.
@@ -59,7 +61,8 @@ constexpr int kCtaGroupAuto = 0;
 // Host-side planner (pure arithmetic, no CUDA calls).  `pair_units` is the number of CTA
 // pairs the device can keep resident (<= num_sms / 2; 0: pairs unavailable).
 ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t pair_units,
-                          int32_t cta_group = kCtaGroupAuto, int32_t chunk_kblocks = kDefaultChunkKBlocks);
+                          int32_t cta_group = kCtaGroupAuto, int32_t chunk_kblocks = kDefaultChunkKBlocks,
+                          bool adaptive = true);
 size_t plan_workspace_bytes(const ScorePlan& p);
 
 // Work unit `unit` in wave `wave`: returns false when the unit idles in that wave.
@@ -91,6 +94,7 @@ struct specs_ctx {
     int engine = SPECS_ENGINE_TCGEN05;
     int pair_units = 0;                    // resident CTA pairs of the pair kernel (0: not available)
     int chunk_kblocks = specs::kDefaultChunkKBlocks;   // see specs_set_accum_chunk
+    bool accum_adaptive = true;
     uint32_t* d_status = nullptr;          // device status word (SPECS_DEV_* bits)
     specs::EncodeTiledFn encode_tiled = nullptr;
     // grow-only device arena for specs_beam_step_host

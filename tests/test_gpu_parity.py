@@ -321,3 +321,63 @@ def test_beam_step_host_equals_device_calls(ctx):
         ctx.specs_beam_step_host(x.hidden, w_dev, x.token_ids, bad, x.cand_offsets, x.draft_tok_logprob, x.reward,
                                  x.uniforms, 1.5, 0.55, tok, blk, wts, cho, acc)
     assert e.value.status == 5
+
+
+# ------------------------------------------------------------------------------- adaptive accumulation chunks
+
+def _score_only(ctx, x):
+    s = DeviceStep(ctx, x)
+    s.score()
+    torch.cuda.synchronize()
+    return s.tok_lp.cpu().numpy()
+
+
+@pytest.mark.parametrize("sigma_z", [1.5, 3.0, 6.0, 12.0])
+def test_adaptive_chunks_keep_the_tolerance_across_logit_magnitudes(ctx, sigma_z):
+    # long reduction (d = 5120), runs of at least three vocabulary tiles per work unit, and logit scales
+    # that land in different chunk lengths (unchunked ... 1024 elements ... the 512-element base)
+    d, V = 5120, 60000
+    cfg = small_config("adapt", (75, 75), 1, 4, d, V, seed=5200 + int(10 * sigma_z), w_sigma=sigma_z / math.sqrt(d))
+    x = I.make_step_inputs(cfg)
+    p = binding.score_plan(x.rows, d, V, ctx.sm_count())
+    runs = [ne - nb for mt, nb, ne in (binding.score_plan_unit(x.rows, d, V, ctx.sm_count(), 0, c)
+                                        for c in range(p["grid"])) if mt >= 0]
+    assert min(runs) >= 3, "the case must exercise the adaptive path"
+    want = O.token_logprobs(x.hidden, x.w_vocab, x.token_ids)
+    got = {}
+    for mode in (binding.ACCUM_ADAPTIVE, 512):
+        ctx.set_accum_chunk(mode)
+        try:
+            got[mode] = _score_only(ctx, x)
+        finally:
+            ctx.set_accum_chunk(binding.ACCUM_ADAPTIVE)
+        assert ctx.device_status() == 0
+        err = np.abs(got[mode] - want).max()
+        assert err <= TOK_ATOL, (mode, err)
+    # the lengthened chunks stay within a quarter of the tolerance of the fixed short ones
+    assert np.abs(got[binding.ACCUM_ADAPTIVE] - got[512]).max() <= TOK_ATOL / 4
+
+
+def test_adaptive_chunks_flag_logits_beyond_the_sampled_magnitude(ctx):
+    # vocabulary entries from the second tile on are 128 times larger than the first tile's: the chunk
+    # length chosen from the first tile is too long for them, which the advisory status bit reports
+    d, V = 5120, 60000
+    cfg = small_config("adapt_surprise", (64, 64), 1, 4, d, V, seed=5300, w_sigma=1.0 / math.sqrt(d))
+    x = I.make_step_inputs(cfg)
+    w = x.w_vocab.copy()
+    big = w[256:]
+    nz = (big & 0x7f80) != 0
+    big[nz] += np.uint16(7 << 7)                             # exponent + 7: exact multiplication by 128
+    x.w_vocab = w
+    want = O.token_logprobs(x.hidden, x.w_vocab, x.token_ids)
+    got = _score_only(ctx, x)
+    assert np.all(np.isfinite(got))
+    assert np.abs(got - want).max() <= 2e-2                  # still close: the bias is a few 1e-3 at most
+    assert ctx.device_status() == binding.DEV_ACCUM_RANGE
+    ctx.set_accum_chunk(512)
+    try:
+        got = _score_only(ctx, x)
+    finally:
+        ctx.set_accum_chunk(binding.ACCUM_ADAPTIVE)
+    assert ctx.device_status() == 0
+    assert np.abs(got - want).max() <= TOK_ATOL
