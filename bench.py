@@ -2,8 +2,9 @@
 """Benchmark of the block-scoring step: scored draft tokens per second.
 
 One *step* is one pass of the whole hot path over one batch of synthetic input:
-LM-head scoring of every drafted token (tcgen05 kernel + split merge), block sums
-of target and generator log-probabilities, SubSample with the fused switch test.
+LM-head scoring of every drafted token (tcgen05 kernel), then one kernel that merges
+the vocabulary splits, sums target and generator log-probabilities per block and runs
+SubSample with the switch test (specs_beam_step).
 The default workload is the 7B-target-shaped single step (1 problem, 16 blocks of
 64 tokens, d = 3584, V = 151936).
 
@@ -36,7 +37,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM bytes (read + write) of one launch of the scoring kernel, from the ncu capture summarised
 # under profiles/ (null until a capture for that workload exists).
-NCU_TRAFFIC_BYTES = {"step7b": 1.0966e9 + 3.7e6}   # profiles/score_tiles_kernel_step7b.md
+NCU_TRAFFIC_BYTES = {"step7b": 1.1071e9 + 3.8e6}   # profiles/score_tiles_pair_kernel_step7b.md
 
 
 def load_peaks():
@@ -218,12 +219,11 @@ def main():
     chosen = torch.empty(P, dtype=torch.int32, device=dev)
     accept = torch.empty(P, dtype=torch.uint8, device=dev)
     ws = torch.empty(ctx.score_workspace_bytes(rows, d, V), dtype=torch.uint8, device=dev)
-    launches_per_step = 5   # score tiles, split merge, target block sums, generator block sums, SubSample+switch
+    launches_per_step = 2   # score tiles; finish (split merge, target and generator block sums, SubSample + switch)
 
     def step():
-        ctx.specs_score_blocks(hidden, w_vocab, ids, boff, tok, None, blk64, ws)
-        ctx.specs_block_sums(draft, boff, None, gen64)
-        ctx.specs_subsample(blk64, gen64, reward, coff, beta, uni, chosen, wts, tau, accept)
+        ctx.specs_beam_step(hidden, w_vocab, ids, boff, coff, draft, reward, uni, beta, tau, tok, blk64, gen64, wts,
+                            chosen, accept, ws)
 
     def barrier():
         if world > 1:
@@ -295,7 +295,9 @@ def main():
         flops = 2.0 * rows * d * V
         achieved = flops / (kernel_ms * 1e-3) / 1e12 if kernel_ms > 0 else None
         peak = peaks["bf16_tflops_sustained"]
-        roofline = {"bound": "tensor", "kernel": "score_tiles_kernel", "achieved": achieved, "peak": peak,
+        plan = binding.score_plan(rows, d, V, ctx.sm_count())
+        roofline = {"bound": "tensor",
+                    "kernel": "score_tiles_pair_kernel" if plan["cta_group"] == 2 else "score_tiles_kernel", "achieved": achieved, "peak": peak,
                     "unit": "TFLOP/s", "frac": achieved / peak if achieved else None,
                     "peak_kind": f"bf16 sustained, of {peaks['source']} (kernel timed inside a long loop)",
                     "frac_of_burst": achieved / peaks["bf16_tflops"] if achieved else None,

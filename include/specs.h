@@ -180,6 +180,33 @@ int specs_subsample_f64(specs_ctx* ctx, const double* blk_lp_target, const doubl
 int specs_accept(specs_ctx* ctx, const float* reward, const int32_t* cand_offsets, int32_t P,
                  float tau, uint8_t* accept, void* cuda_stream);
 
+/* One whole beam step on DEVICE buffers in two launches: the LM-head scoring
+ * kernel, then one kernel that, per problem, merges the vocabulary splits into
+ * log pi_target of every drafted token (Section 2, Appendix E.3), sums target and
+ * generator log-probabilities per drafted block (Eq. 1), draws SubSample's
+ * candidate (Algorithm 2) and evaluates the switch test (Algorithm 1, Step III).
+ * Results are identical to specs_score_blocks + specs_block_sums +
+ * specs_subsample_f64 on the same inputs; only the launch count differs.
+ *
+ *   gen_tok_logprob  float [rows]: the generator's own per-token log-probabilities
+ *                    (NULL: pi_gen = pi_target, S_i = beta * reward[i]).
+ *   blk_logprob_f64  double [B] out, required: block sums of log pi_target.
+ *   gen_blk_logprob_f64 double [B] out, required when gen_tok_logprob is given.
+ *   weights, accept  may be NULL.  chosen int32 [P] out, required.
+ *   workspace        as for specs_score_blocks.
+ * Other arguments as in specs_score_blocks and specs_subsample.  The rows of a
+ * problem must be contiguous, which the two offset arrays imply.  Tensor-core
+ * engines only (SPECS_ERR_SHAPE if the SIMT aid is selected).  One CTA handles one
+ * problem, so a single problem with very many rows (beyond about 10^5) is better
+ * served by the separate calls. */
+int specs_beam_step(specs_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* token_ids,
+                    const int64_t* block_offsets, const int32_t* cand_offsets,
+                    const float* gen_tok_logprob, const float* reward, const float* uniforms,
+                    int64_t rows, int32_t d, int32_t V, int32_t B, int32_t P, float beta, float tau,
+                    float* tok_logprob, double* blk_logprob_f64, double* gen_blk_logprob_f64,
+                    float* weights, int32_t* chosen, uint8_t* accept,
+                    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Synchronise `cuda_stream`, return the device status word (a combination of
  * SPECS_DEV_* bits, 0 if clean) through *h_bits and clear it.  Returns
  * SPECS_ERR_DEVICE_TIMEOUT / SPECS_ERR_TOKEN_RANGE (timeout first) when a bit is
@@ -187,9 +214,8 @@ int specs_accept(specs_ctx* ctx, const float* reward, const int32_t* cand_offset
 int specs_device_status(specs_ctx* ctx, uint32_t* h_bits, void* cuda_stream);
 
 /* One whole beam step from HOST buffers (the end-to-end path): copies the step's
- * inputs to the device, runs specs_score_blocks, specs_block_sums on the
- * generator's per-token log-probabilities, and specs_subsample_f64 with the switch
- * test, copies the results back and synchronises the stream before returning.
+ * inputs to the device, runs specs_beam_step, copies the results back and
+ * synchronises the stream before returning.
  * W_vocab is the model's weight and stays a DEVICE pointer.  The context keeps
  * grow-only device and pinned staging buffers for this call, so it may allocate on
  * first use or when sizes grow.  h_block_offsets and h_cand_offsets are validated

@@ -44,6 +44,8 @@ SIGNATURES = {
     "specs_subsample": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _f32, _vp, _vp, _vp, _f32, _vp, _vp]),
     "specs_subsample_f64": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _f32, _vp, _vp, _vp, _f32, _vp, _vp]),
     "specs_accept": (C.c_int, [_vp, _vp, _vp, _i32, _f32, _vp, _vp]),
+    "specs_beam_step": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _f32, _f32,
+                                  _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_size_t, _vp]),
     "specs_device_status": (C.c_int, [_vp, C.POINTER(C.c_uint32), _vp]),
     "specs_beam_step_host": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32,
                                        _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -201,6 +203,21 @@ class Context:
         P = cand_offsets.shape[0] - 1
         _check(self._lib.specs_accept(self._h, _ptr(reward), _ptr(cand_offsets), P, float(tau), _ptr(accept),
                                       _stream()), "specs_accept")
+
+    def specs_beam_step(self, hidden, w_vocab, token_ids, block_offsets, cand_offsets, gen_tok_logprob, reward,
+                        uniforms, beta, tau, tok_logprob, blk_logprob_f64, gen_blk_logprob_f64, weights, chosen,
+                        accept, workspace):
+        """The whole step on device tensors in two launches (scoring kernel + per-problem finish kernel)."""
+        rows, d = hidden.shape
+        V = w_vocab.shape[0]
+        B = block_offsets.shape[0] - 1
+        P = cand_offsets.shape[0] - 1
+        _check(self._lib.specs_beam_step(
+            self._h, _ptr(hidden), _ptr(w_vocab), _ptr(token_ids), _ptr(block_offsets), _ptr(cand_offsets),
+            _ptr(gen_tok_logprob), _ptr(reward), _ptr(uniforms), rows, d, V, B, P, float(beta), float(tau),
+            _ptr(tok_logprob), _ptr(blk_logprob_f64), _ptr(gen_blk_logprob_f64), _ptr(weights), _ptr(chosen),
+            _ptr(accept), _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
+            _stream()), "specs_beam_step")
 
     def specs_beam_step_host(self, h_hidden, w_vocab, h_token_ids, h_block_offsets, h_cand_offsets,
                              h_gen_tok_logprob, h_reward, h_uniforms, beta, tau,

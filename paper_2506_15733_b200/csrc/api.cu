@@ -347,6 +347,41 @@ int specs_accept(specs_ctx* ctx, const float* reward, const int32_t* cand_offset
     return launch_accept(reward, cand_offsets, P, tau, accept, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int specs_beam_step(specs_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* token_ids,
+                    const int64_t* block_offsets, const int32_t* cand_offsets, const float* gen_tok_logprob,
+                    const float* reward, const float* uniforms, int64_t rows, int32_t d, int32_t V, int32_t B,
+                    int32_t P, float beta, float tau, float* tok_logprob, double* blk_logprob_f64,
+                    double* gen_blk_logprob_f64, float* weights, int32_t* chosen, uint8_t* accept, void* workspace,
+                    size_t workspace_bytes, void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    int st = check_score_shapes(rows, d, V, B);
+    if (st != SPECS_OK) return st;
+    if (P < 0) return SPECS_ERR_SHAPE;
+    if (P == 0) return SPECS_OK;
+    if (!W_vocab || !block_offsets || !cand_offsets || !chosen) return SPECS_ERR_NULL;
+    if (rows > 0 && (!hidden || !token_ids || !tok_logprob || !workspace)) return SPECS_ERR_NULL;
+    if (B > 0 && (!reward || !uniforms || !blk_logprob_f64 || (gen_tok_logprob && !gen_blk_logprob_f64)))
+        return SPECS_ERR_NULL;
+    if (!aligned16(hidden) || !aligned16(W_vocab) || !aligned16(workspace)) return SPECS_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+    if (ctx->engine == SPECS_ENGINE_SIMT) return SPECS_ERR_SHAPE;         // the fused step is tensor-core only
+
+    const int cta_group = ctx->engine == SPECS_ENGINE_TCGEN05_1CTA ? 1
+                        : ctx->engine == SPECS_ENGINE_TCGEN05_2CTA ? 2 : kCtaGroupAuto;
+    const ScorePlan plan = make_score_plan(rows, d, V, ctx->num_sms, ctx->pair_units, cta_group, ctx->chunk_kblocks,
+                                           ctx->accum_adaptive);
+    if (rows > 0) {
+        if (workspace_bytes < plan_workspace_bytes(plan)) return SPECS_ERR_WORKSPACE;
+        st = launch_score_tcgen05(ctx, plan, hidden, W_vocab, token_ids, static_cast<float*>(workspace), stream);
+        if (st != SPECS_OK) return st;
+    }
+    return launch_finish_step(ctx, plan, static_cast<const float*>(workspace), token_ids, block_offsets, cand_offsets,
+                              P, gen_tok_logprob, reward, uniforms, beta, tau, tok_logprob, blk_logprob_f64,
+                              gen_blk_logprob_f64, weights, chosen, accept, stream);
+}
+
 int specs_device_status(specs_ctx* ctx, uint32_t* h_bits, void* cuda_stream) {
     if (!ctx) return SPECS_ERR_NULL;
     DeviceGuard guard(ctx->device);
@@ -436,22 +471,14 @@ int specs_beam_step_host(specs_ctx* ctx, const void* h_hidden, const void* W_voc
     if (ok && h_gen_tok_logprob) ok = h2d(o_gen, h_gen_tok_logprob, (size_t)rows * 4);
     if (!ok) return SPECS_ERR_CUDA;
 
-    st = specs_score_blocks(ctx, A + o_hidden, W_vocab, reinterpret_cast<int32_t*>(A + o_ids),
-                            reinterpret_cast<int64_t*>(A + o_boff), rows, d, V, B,
-                            reinterpret_cast<float*>(A + o_tok), nullptr, reinterpret_cast<double*>(A + o_blk_t),
-                            A + o_ws, ws_bytes, cuda_stream);
-    if (st != SPECS_OK) return st;
-    const double* gen_blk = nullptr;
-    if (h_gen_tok_logprob) {
-        st = specs_block_sums(ctx, reinterpret_cast<float*>(A + o_gen), reinterpret_cast<int64_t*>(A + o_boff), B,
-                              nullptr, reinterpret_cast<double*>(A + o_blk_g), cuda_stream);
-        if (st != SPECS_OK) return st;
-        gen_blk = reinterpret_cast<double*>(A + o_blk_g);
-    }
-    st = specs_subsample_f64(ctx, reinterpret_cast<double*>(A + o_blk_t), gen_blk, reinterpret_cast<float*>(A + o_rew),
-                             reinterpret_cast<int32_t*>(A + o_coff), P, beta, reinterpret_cast<float*>(A + o_uni),
-                             reinterpret_cast<int32_t*>(A + o_cho), reinterpret_cast<float*>(A + o_wts), tau,
-                             reinterpret_cast<uint8_t*>(A + o_acc), cuda_stream);
+    st = specs_beam_step(ctx, A + o_hidden, W_vocab, reinterpret_cast<int32_t*>(A + o_ids),
+                         reinterpret_cast<int64_t*>(A + o_boff), reinterpret_cast<int32_t*>(A + o_coff),
+                         h_gen_tok_logprob ? reinterpret_cast<float*>(A + o_gen) : nullptr,
+                         reinterpret_cast<float*>(A + o_rew), reinterpret_cast<float*>(A + o_uni), rows, d, V, B, P,
+                         beta, tau, reinterpret_cast<float*>(A + o_tok), reinterpret_cast<double*>(A + o_blk_t),
+                         reinterpret_cast<double*>(A + o_blk_g), reinterpret_cast<float*>(A + o_wts),
+                         reinterpret_cast<int32_t*>(A + o_cho), reinterpret_cast<uint8_t*>(A + o_acc), A + o_ws,
+                         ws_bytes, cuda_stream);
     if (st != SPECS_OK) return st;
     ok = d2h(h_tok_logprob, o_tok, (size_t)rows * 4) && d2h(h_blk_logprob, o_blk_t, (size_t)B * 8) &&
          d2h(h_weights, o_wts, (size_t)B * 4) && d2h(h_chosen, o_cho, (size_t)P * 4) &&

@@ -6,7 +6,8 @@
 //   subsample_kernel      one warp per problem: scores of Eq. (1), the normalised weights of
 //                         Algorithm 2, a Gumbel-max draw from caller-supplied uniforms and the
 //                         switch test of Algorithm 1, Step III;
-//   accept_kernel         the switch test alone.
+//   accept_kernel         the switch test alone;
+//   finish_step_kernel    all of the above for one problem per CTA, for the fused beam step.
 #include "specs_internal.h"
 
 namespace specs {
@@ -21,21 +22,14 @@ constexpr unsigned kFull = 0xffffffffu;
 // base-2 units (max logit * log2 e), the sum of 2^(logit*log2e - max) over that half of the CTA's
 // vocabulary chunk, and the drafted id's logit if the id fell there (-inf otherwise).  A half
 // that saw no valid column (vocabulary tail) carries max = -inf, sum = 0.
-constexpr int kMergeWarps = 8;                              // warps per block: each takes every 8th split
+constexpr int kMergeBatch = 6;                              // splits whose six floats are loaded before any is used
 
-__global__ void __launch_bounds__(32 * kMergeWarps)
-merge_splits_kernel(const ScorePlan plan, const float* __restrict__ workspace,
-                    const int32_t* __restrict__ token_ids, float* __restrict__ tok_logprob,
-                    uint32_t* __restrict__ status) {
-    // A block owns 32 consecutive rows (lane = row, so loads are coalesced); its warps share the
-    // vocabulary splits of those rows and combine their partial (max, sum, logit) in shared memory.
-    __shared__ float sh_max[kMergeWarps][32], sh_logit[kMergeWarps][32];
-    __shared__ double sh_sum[kMergeWarps][32];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t row = (int64_t)blockIdx.x * 32 + lane;
-    const bool live = row < plan.rows;
-    const int64_t row_c = live ? row : plan.rows - 1;
-    const int mt = (int)(row_c / kBlockM), r = (int)(row_c % kBlockM);
+// log pi_target of the drafted token of `row`: fold the row's per-split partials, in split order,
+// into (max, sum) in base-2 units, then  logit - (max + log2 sum) * ln 2.  The loads of a batch of
+// splits are independent of the arithmetic and of each other, so a batch costs one trip to L2.
+__device__ __forceinline__ float merged_logprob(const ScorePlan& plan, const float* __restrict__ workspace,
+                                                int64_t row, int32_t id, uint32_t* __restrict__ status) {
+    const int mt = (int)(row / kBlockM), r = (int)(row % kBlockM);
     // the row tile's work unit: super tile (cta_group row tiles) and the CTA's rank inside the unit
     const int cg = plan.cta_group, sup = mt / cg, rank = mt % cg;
     int wave, i, gm, splits;
@@ -51,40 +45,45 @@ merge_splits_kernel(const ScorePlan plan, const float* __restrict__ workspace,
 
     float m = -INFINITY, logit = -INFINITY;
     double sum = 0.0;
-    for (int s = warp; s < splits; s += kMergeWarps) {
-        const float* p = base + s * stride;
-        const float m0 = p[0], s0 = p[kBlockM], t0 = p[2 * kBlockM];
-        const float m1 = p[kHalf], s1 = p[kHalf + kBlockM], t1 = p[kHalf + 2 * kBlockM];
-        const float mn = fmaxf(m, fmaxf(m0, m1));
-        if (mn != -INFINITY) {
-            // exp2f(-inf) = 0 takes care of halves and states that have seen nothing yet
-            sum = sum * (double)exp2f(m - mn) + (double)s0 * (double)exp2f(m0 - mn) +
-                  (double)s1 * (double)exp2f(m1 - mn);
-            m = mn;
+    for (int s0 = 0; s0 < splits; s0 += kMergeBatch) {
+        float v[kMergeBatch][6];
+#pragma unroll
+        for (int u = 0; u < kMergeBatch; ++u) {
+            const bool live = s0 + u < splits;
+            const float* p = base + (size_t)(live ? s0 + u : s0) * stride;
+            const float m0 = __ldcg(p), s_0 = __ldcg(p + kBlockM), t0 = __ldcg(p + 2 * kBlockM);
+            const float m1 = __ldcg(p + kHalf), s_1 = __ldcg(p + kHalf + kBlockM), t1 = __ldcg(p + kHalf + 2 * kBlockM);
+            v[u][0] = live ? m0 : -INFINITY; v[u][1] = live ? s_0 : 0.0f; v[u][2] = live ? t0 : -INFINITY;
+            v[u][3] = live ? m1 : -INFINITY; v[u][4] = live ? s_1 : 0.0f; v[u][5] = live ? t1 : -INFINITY;
         }
-        logit = fmaxf(logit, fmaxf(t0, t1));
-    }
-    sh_max[warp][lane] = m; sh_sum[warp][lane] = sum; sh_logit[warp][lane] = logit;
-    __syncthreads();
-    if (warp != 0 || !live) return;
-    float gmax = sh_max[0][lane];
 #pragma unroll
-    for (int w = 1; w < kMergeWarps; ++w) gmax = fmaxf(gmax, sh_max[w][lane]);
-    double total = 0.0;
-    float picked = -INFINITY;
-#pragma unroll
-    for (int w = 0; w < kMergeWarps; ++w) {
-        if (sh_max[w][lane] != -INFINITY) total += sh_sum[w][lane] * (double)exp2f(sh_max[w][lane] - gmax);
-        picked = fmaxf(picked, sh_logit[w][lane]);
+        for (int u = 0; u < kMergeBatch; ++u) {
+            const float mn = fmaxf(m, fmaxf(v[u][0], v[u][3]));
+            if (mn != -INFINITY) {
+                // exp2f(-inf) = 0 takes care of halves and states that have seen nothing yet
+                sum = sum * (double)exp2f(m - mn) + (double)v[u][1] * (double)exp2f(v[u][0] - mn) +
+                      (double)v[u][4] * (double)exp2f(v[u][3] - mn);
+                m = mn;
+            }
+            logit = fmaxf(logit, fmaxf(v[u][2], v[u][5]));
+        }
     }
-    const int32_t id = token_ids[row];
     if (id < 0 || id >= plan.V) {
-        tok_logprob[row] = __int_as_float(0x7fc00000);      // no such vocabulary entry: NaN
         atomicOr(status, SPECS_DEV_TOKEN_RANGE);
-        return;
+        return __int_as_float(0x7fc00000);                  // no such vocabulary entry: NaN
     }
-    const double lse = ((double)gmax + log2(total)) * kLn2; // natural-log normaliser
-    tok_logprob[row] = (float)((double)picked - lse);
+    const double lse = ((double)m + log2(sum)) * kLn2;      // natural-log normaliser
+    return (float)((double)logit - lse);
+}
+
+__global__ void __launch_bounds__(128)
+merge_splits_kernel(const ScorePlan plan, const float* __restrict__ workspace,
+                    const int32_t* __restrict__ token_ids, float* __restrict__ tok_logprob,
+                    uint32_t* __restrict__ status) {
+    // one thread per row; consecutive lanes read consecutive floats of a slot
+    const int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= plan.rows) return;
+    tok_logprob[row] = merged_logprob(plan, workspace, row, token_ids[row], status);
 }
 
 // ------------------------------------------------------------------------------------ block sums
@@ -112,16 +111,13 @@ __device__ __forceinline__ double score_of(const LP* lp_t, const LP* lp_g, const
     return __dadd_rn(__dsub_rn((double)lp_t[i], (double)lp_g[i]), br);
 }
 
+// One warp, one problem with candidates [a, b): scores, weights, Gumbel-max pick, switch test.
 template <typename LP>
-__global__ void subsample_kernel(const LP* __restrict__ lp_t, const LP* __restrict__ lp_g,
-                                 const float* __restrict__ reward, const int32_t* __restrict__ cand_offsets,
-                                 int32_t P, float beta, const float* __restrict__ uniforms,
-                                 int32_t* __restrict__ chosen, float* __restrict__ weights, float tau,
-                                 uint8_t* __restrict__ accept) {
-    const int p = (int)(((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
-    const int lane = threadIdx.x & 31;
-    if (p >= P) return;
-    const int a = cand_offsets[p], b = cand_offsets[p + 1];
+__device__ __forceinline__ void subsample_problem(const LP* lp_t, const LP* lp_g, const float* __restrict__ reward,
+                                                  int a, int b, int p, int lane, float beta,
+                                                  const float* __restrict__ uniforms, int32_t* __restrict__ chosen,
+                                                  float* __restrict__ weights, float tau,
+                                                  uint8_t* __restrict__ accept) {
     if (b <= a) {
         if (lane == 0) {
             if (chosen) chosen[p] = -1;
@@ -166,6 +162,67 @@ __global__ void subsample_kernel(const LP* __restrict__ lp_t, const LP* __restri
     }
 }
 
+template <typename LP>
+__global__ void subsample_kernel(const LP* __restrict__ lp_t, const LP* __restrict__ lp_g,
+                                 const float* __restrict__ reward, const int32_t* __restrict__ cand_offsets,
+                                 int32_t P, float beta, const float* __restrict__ uniforms,
+                                 int32_t* __restrict__ chosen, float* __restrict__ weights, float tau,
+                                 uint8_t* __restrict__ accept) {
+    const int p = (int)(((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+    const int lane = threadIdx.x & 31;
+    if (p >= P) return;
+    subsample_problem<LP>(lp_t, lp_g, reward, cand_offsets[p], cand_offsets[p + 1], p, lane, beta, uniforms, chosen,
+                          weights, tau, accept);
+}
+
+// ------------------------------------------------------------------------------------ fused finish
+// Everything after the LM-head pass for one problem per CTA: merge the vocabulary splits of the
+// problem's rows, sum target and generator log-probabilities per drafted block, then SubSample and
+// the switch test on those sums.  The three phases are separated by CTA barriers; the block sums
+// travel through the output arrays blk_lp / gen_lp (double).  One launch instead of four.
+constexpr int kFinishThreads = 1024;
+
+__global__ void __launch_bounds__(kFinishThreads)
+finish_step_kernel(const ScorePlan plan, const float* __restrict__ workspace, const int32_t* __restrict__ token_ids,
+                   const int64_t* __restrict__ block_offsets, const int32_t* __restrict__ cand_offsets,
+                   const float* __restrict__ gen_tok_logprob, const float* __restrict__ reward,
+                   const float* __restrict__ uniforms, float beta, float tau, float* __restrict__ tok_logprob,
+                   double* blk_lp, double* gen_lp, float* __restrict__ weights, int32_t* __restrict__ chosen,
+                   uint8_t* __restrict__ accept, uint32_t* __restrict__ status) {
+    // Launched with programmatic stream serialisation: wait here for the scoring kernel's results.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int p = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int a = cand_offsets[p], b = cand_offsets[p + 1];
+    if (b > a) {
+        const int64_t row_a = block_offsets[a], row_b = block_offsets[b];   // the problem's rows are contiguous
+        for (int64_t row = row_a + threadIdx.x; row < row_b; row += kFinishThreads)
+            tok_logprob[row] = merged_logprob(plan, workspace, row, token_ids[row], status);
+        __syncthreads();
+        for (int i = a + warp; i < b; i += kFinishThreads / 32) {
+            const int64_t t0 = block_offsets[i], t1 = block_offsets[i + 1];
+            double lp = 0.0, lq = 0.0;
+            for (int64_t t = t0 + lane; t < t1; t += 32) {
+                lp += (double)tok_logprob[t];
+                if (gen_tok_logprob) lq += (double)gen_tok_logprob[t];
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                lp += __shfl_xor_sync(kFull, lp, o);
+                lq += __shfl_xor_sync(kFull, lq, o);
+            }
+            if (lane == 0) {
+                blk_lp[i] = lp;
+                if (gen_tok_logprob) gen_lp[i] = lq;
+            }
+        }
+        __syncthreads();
+    }
+    if (warp == 0)
+        subsample_problem<double>(blk_lp, gen_tok_logprob ? gen_lp : nullptr, reward, a, b, p, lane, beta, uniforms,
+                                  chosen, weights, tau, accept);
+}
+
 __global__ void accept_kernel(const float* __restrict__ reward, const int32_t* __restrict__ cand_offsets, int32_t P,
                               float tau, uint8_t* __restrict__ accept) {
     const int p = (int)(((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
@@ -189,10 +246,30 @@ inline unsigned warps_grid(int64_t warps, int threads) {
 int launch_merge(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, const int32_t* token_ids,
                  float* tok_logprob, cudaStream_t stream) {
     if (plan.rows == 0) return SPECS_OK;
-    const unsigned blocks = (unsigned)((plan.rows + 31) / 32);
-    merge_splits_kernel<<<blocks, 32 * kMergeWarps, 0, stream>>>(plan, workspace, token_ids, tok_logprob,
-                                                                 ctx->d_status);
+    const unsigned blocks = (unsigned)((plan.rows + 127) / 128);
+    merge_splits_kernel<<<blocks, 128, 0, stream>>>(plan, workspace, token_ids, tok_logprob, ctx->d_status);
     return cuda_status(cudaGetLastError());
+}
+
+int launch_finish_step(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, const int32_t* token_ids,
+                       const int64_t* block_offsets, const int32_t* cand_offsets, int32_t P,
+                       const float* gen_tok_logprob, const float* reward, const float* uniforms, float beta, float tau,
+                       float* tok_logprob, double* blk_lp, double* gen_lp, float* weights, int32_t* chosen,
+                       uint8_t* accept, cudaStream_t stream) {
+    if (P == 0) return SPECS_OK;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)P, 1, 1);
+    cfg.blockDim = dim3(kFinishThreads, 1, 1);
+    cfg.stream = stream;
+    // the launch is set up while the scoring kernel still runs; the kernel itself waits for it
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cuda_status(cudaLaunchKernelEx(&cfg, finish_step_kernel, plan, workspace, token_ids, block_offsets,
+                                          cand_offsets, gen_tok_logprob, reward, uniforms, beta, tau, tok_logprob,
+                                          blk_lp, gen_lp, weights, chosen, accept, ctx->d_status));
 }
 
 int launch_block_sums(const float* per_token, const int64_t* block_offsets, int32_t B, float* out, double* out_f64,

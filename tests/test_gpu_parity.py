@@ -298,6 +298,63 @@ def test_block_sums_kernel(ctx):
         np.abs(o32.cpu().numpy() - want).max() <= 1e-6 * np.abs(want).max()
 
 
+# ------------------------------------------------------------------------------- fused device step
+
+def _fused_step(ctx, s, beta, tau, with_draft=True):
+    ctx.specs_beam_step(s.hidden, s.w_vocab, s.token_ids, s.block_offsets, s.cand_offsets,
+                        s.draft if with_draft else None, s.reward, s.uniforms, beta, tau, s.tok_lp, s.blk_lp64,
+                        s.gen_blk64 if with_draft else None, s.weights, s.chosen, s.accept, s.workspace)
+    torch.cuda.synchronize()
+    return s.results()
+
+
+@pytest.mark.parametrize("engine", [binding.ENGINE_TCGEN05] + TC_ENGINES)
+@pytest.mark.parametrize("with_draft", [True, False])
+def test_fused_beam_step_equals_the_separate_calls(ctx, engine, with_draft):
+    cfg = small_config("fused", (3, 90), 7, 5, 256, 2500, seed=4950)
+    x = I.make_step_inputs(cfg)
+    # holes: an empty block, an empty problem in the middle and one at the end
+    lens = np.diff(x.block_offsets)
+    lens[4] = 0
+    x.block_offsets = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    rows = int(x.block_offsets[-1])
+    x.hidden, x.token_ids, x.draft_tok_logprob = x.hidden[:rows], x.token_ids[:rows], x.draft_tok_logprob[:rows]
+    x.cand_offsets = np.array([0, 5, 10, 10, 15, 20, 25, 35, 35], dtype=np.int32)
+    ctx.set_engine(engine)
+    try:
+        want = DeviceStep(ctx, x).step(1.5, 0.55, with_draft)
+        got = _fused_step(ctx, DeviceStep(ctx, x), 1.5, 0.55, with_draft)
+    finally:
+        ctx.set_engine(binding.ENGINE_TCGEN05)
+    for key in ("tok_logprob", "blk_logprob_f64", "weights", "chosen", "accept") + (("blk_logprob_gen",) if with_draft else ()):
+        assert np.array_equal(got[key], want[key]), key
+    assert got["chosen"][2] == -1 and got["chosen"][7] == -1 and got["accept"][2] == 0
+    ref = oracle_step(x, 1.5, 0.55, with_draft)
+    got["blk_logprob"] = got["blk_logprob_f64"].astype(np.float32)
+    assert_step_matches(got, ref, x.cand_offsets, x.block_offsets)
+    assert ctx.device_status() == 0
+
+
+def test_fused_beam_step_flags_bad_ids_and_validates(ctx):
+    cfg = small_config("fused_bad", (8, 8), 2, 2, 64, 300, seed=4960)
+    x = I.make_step_inputs(cfg)
+    x.token_ids = x.token_ids.copy()
+    x.token_ids[5] = 999
+    s = DeviceStep(ctx, x)
+    got = _fused_step(ctx, s, 1.0, 0.5)
+    assert np.isnan(got["tok_logprob"][5]) and np.isfinite(np.delete(got["tok_logprob"], 5)).all()
+    assert ctx.device_status() == binding.DEV_TOKEN_RANGE
+    with pytest.raises(binding.SpecsError) as e:
+        ctx.specs_beam_step(s.hidden, s.w_vocab, s.token_ids, s.block_offsets, s.cand_offsets, s.draft, s.reward,
+                            s.uniforms, 1.0, 0.5, s.tok_lp, None, s.gen_blk64, s.weights, s.chosen, s.accept, s.workspace)
+    assert e.value.status == 1                                # the block sums are required outputs
+    with pytest.raises(binding.SpecsError) as e:
+        ctx.specs_beam_step(s.hidden, s.w_vocab, s.token_ids, s.block_offsets, s.cand_offsets, s.draft, s.reward,
+                            s.uniforms, 1.0, 0.5, s.tok_lp, s.blk_lp64, s.gen_blk64, s.weights, s.chosen, s.accept,
+                            s.workspace[:64])
+    assert e.value.status == 4
+
+
 # ------------------------------------------------------------------------------- host-buffer entry point
 
 def test_beam_step_host_equals_device_calls(ctx):
