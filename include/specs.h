@@ -280,9 +280,10 @@ int specs_score_plan_unit(int64_t rows, int32_t d, int32_t V, int32_t num_sms, i
  *
  * Limits and sharing:
  *   - the plan for (rows, d, V) must fit the fixed scratch (waves x SMs x 3072 bytes
- *     <= SPECS_NOALLOC_SCRATCH_BYTES; about 110 000 rows at d = 3584 and 85 000 at
- *     d = 5120 on a 148-SM part); larger problems return SPECS_ERR_LIMIT and launch
- *     nothing.  Split the rows over several calls instead.
+ *     <= SPECS_NOALLOC_SCRATCH_BYTES; roughly 50 000 rows at d = 3584 or 5120 and
+ *     170 000 at d = 1536 on a 148-SM part; specs_score_plan gives the exact size);
+ *     larger problems return SPECS_ERR_LIMIT and launch nothing.  Split the rows over
+ *     several calls instead.
  *   - all calls on a device share the one array, which still holds the previous
  *     call's contents.  Nothing in it has to start at zero (each slot is written
  *     before it is read within a call), but calls whose kernels overlap on the GPU,
