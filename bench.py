@@ -176,11 +176,13 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
 
+    from paper_2506_15733_b200.replicas import Replicas
+    ranks = Replicas.from_env()
+    rank, local_rank, world = ranks.rank, ranks.local_rank, ranks.world
+    if args.impl == "reference" and rank != 0:
+        return                                               # rank 0 alone times the CPU oracle
     from paper_2506_15733_b200 import inputs
     cfg = inputs.CONFIGS[args.config]
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
 
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else args.steps
@@ -192,15 +194,13 @@ def main():
     args.warmup = 50 if args.warmup is None else max(args.warmup, 3)
 
     import torch
-    import torch.distributed as dist
     from paper_2506_15733_b200 import binding
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the scoring path has no CPU fallback")
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+    ranks.init("nccl", torch.device(dev))
 
     x = inputs.make_step_inputs(cfg)
     rows, B, P, d, V = x.rows, x.blocks, cfg.problems, cfg.d, cfg.vocab
@@ -226,8 +226,7 @@ def main():
                             chosen, accept, ws)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        ranks.barrier()
         torch.cuda.synchronize()
 
     for _ in range(args.warmup):
@@ -246,10 +245,7 @@ def main():
     kernel_ms, kernel_launches = ctx.score_kernel_ms()
     ctx.set_timing(False)
     status_bits = ctx.device_status()
-    if world > 1:
-        tm = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-        total_ms = float(tm.item())
+    total_ms = ranks.max_over_ranks(total_ms)
     value = rows * world * args.steps / (total_ms * 1e-3)
 
     # end to end through the host-buffer entry point: pinned host inputs, H2D and D2H inside the timed region
@@ -281,10 +277,7 @@ def main():
             host_step()           # synchronises its stream before returning
         barrier()
         dt = time.perf_counter() - t0
-        if world > 1:
-            tm = torch.tensor([dt], dtype=torch.float64, device=dev)
-            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-            dt = float(tm.item())
+        dt = ranks.max_over_ranks(dt)
         assert torch.equal(o_cho.to(dev), chosen) and torch.equal(o_tok.to(dev), tok), "host path disagrees"
         e2e = {"value": rows * world * e2e_steps / dt, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": e2e_steps,
@@ -321,8 +314,7 @@ def main():
                 "tensor_tflops_whole_step": flops * args.steps / (total_ms * 1e-3) / 1e12}
         print(json.dumps(line))
     ctx.close()
-    if world > 1:
-        dist.destroy_process_group()
+    ranks.shutdown()
 
 
 if __name__ == "__main__":
