@@ -1,0 +1,152 @@
+"""CPU oracle for the selection variants and the Algorithm-1 controller.  TEST INFRASTRUCTURE ONLY.
+
+Same rules as specs_oracle.py: float64 numpy and plain Python loops, the definitions written out,
+nothing imported from the product, never called by it.
+
+What each function follows in the paper:
+
+  select            Algorithm 2 with its candidate set L made explicit (P(i* = i) is proportional to
+                    exp(S_i) * 1(i in L)), plus the selection rules of the systems the paper compares
+                    with (Section 4.1, Baselines): beam search and RSD++ keep the candidate with the
+                    highest PRM score, which is also what Algorithm 2 tends to as beta grows when
+                    the log-ratio is dropped; "SPECS (no LL)" (Section 4.3) drops the log-ratio.
+  switch_flags      Algorithm 1, Step III (some candidate's reward exceeds tau: the draft generates
+                    next); its mirror for "SPECS (pi_draft start)" (Section 4.3: go to the target when
+                    no candidate of the draft exceeds tau); and RSD++'s rule (Section 4.1: if the
+                    reward of the selected draft candidate falls below the threshold, the step is
+                    redone with the target).
+  Controller        Algorithm 1 as a per-problem state machine: which model generates the next
+                    block, appending the selected block, the switch, the stop at the target length;
+                    with the ablation policies of Section 4.3 (only-small generation, random
+                    switching, draft start) and the two baselines (beam search with one model, RSD++).
+
+Readings taken where the paper is silent: the switch test looks at every candidate's reward, masked
+or not; an empty problem (or one whose candidates are all masked) selects -1 and raises no flag;
+ties in the highest reward go to the lowest index; Algorithm 1 only ever assigns pi_gen <- pi_draft,
+while Section 2.3 and the reported share of target steps describe a decision taken at every step:
+`sticky` chooses between the two.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+SELECT_SUBSAMPLE, SELECT_BEST_REWARD = 0, 1
+SCORE_NO_LL = 0x1
+SWITCH_ANY_ABOVE, SWITCH_NONE_ABOVE, SWITCH_CHOSEN_BELOW = 0, 1, 2
+GEN_TARGET, GEN_DRAFT, GEN_DONE = 0, 1, -1
+POLICY_SPECS, POLICY_ONLY_DRAFT, POLICY_ONLY_TARGET, POLICY_RANDOM, POLICY_DRAFT_START, POLICY_RSD = 0, 1, 2, 3, 4, 5
+
+
+def select(lp_target, lp_gen, reward, mask, cand_offsets, beta, uniforms, rule=SELECT_SUBSAMPLE, score_flags=0):
+    """Per problem: the selected candidate (index local to the problem, -1 if none is eligible), the
+    selection weights over the problem's candidates, and the top-two margin of the quantity maximised."""
+    r = np.asarray(reward, dtype=np.float64)
+    B = r.shape[0]
+    beta = float(np.float32(beta))
+    if lp_gen is None or (score_flags & SCORE_NO_LL):
+        S = beta * r
+    else:
+        S = (np.asarray(lp_target, dtype=np.float64) - np.asarray(lp_gen, dtype=np.float64)) + beta * r
+    in_L = np.ones(B, dtype=bool) if mask is None else (np.asarray(mask) != 0)
+    P = len(cand_offsets) - 1
+    chosen = np.full(P, -1, dtype=np.int32)
+    margin = np.full(P, np.inf)
+    w = np.zeros(B)
+    for p in range(P):
+        a, b = int(cand_offsets[p]), int(cand_offsets[p + 1])
+        elig = [i for i in range(a, b) if in_L[i]]
+        if not elig:
+            continue
+        if rule == SELECT_BEST_REWARD:
+            key = {i: r[i] for i in elig}
+        else:
+            u = np.asarray(uniforms, dtype=np.float64)
+            if np.any((u[a:b] <= 0.0) | (u[a:b] >= 1.0)):
+                raise ValueError("uniforms must lie strictly inside (0, 1)")
+            key = {i: S[i] - np.log(-np.log(u[i])) for i in elig}
+        best = elig[0]
+        for i in elig[1:]:
+            if key[i] > key[best]:                    # strict: the lowest index keeps a tie
+                best = i
+        chosen[p] = best - a
+        others = [key[i] for i in elig if i != best]
+        if others:
+            margin[p] = key[best] - max(others)
+        if rule == SELECT_BEST_REWARD:
+            w[best] = 1.0
+        else:
+            m = max(S[i] for i in elig)
+            z = sum(np.exp(S[i] - m) for i in elig)
+            for i in elig:
+                w[i] = np.exp(S[i] - m) / z
+    return chosen, w, margin
+
+
+def switch_flags(reward, cand_offsets, chosen, tau, rule=SWITCH_ANY_ABOVE):
+    r = np.asarray(reward, dtype=np.float32)
+    tau = np.float32(tau)
+    P = len(cand_offsets) - 1
+    out = np.zeros(P, dtype=np.uint8)
+    for p in range(P):
+        a, b = int(cand_offsets[p]), int(cand_offsets[p + 1])
+        if b <= a:
+            continue
+        any_above = bool(np.max(r[a:b]) > tau)
+        if rule == SWITCH_ANY_ABOVE:
+            out[p] = any_above
+        elif rule == SWITCH_NONE_ABOVE:
+            out[p] = not any_above
+        else:
+            out[p] = chosen[p] >= 0 and bool(r[a + int(chosen[p])] < tau)
+    return out
+
+
+class Controller:
+    """Algorithm 1 for P problems.  generators() says who drafts the next n blocks of every problem
+    (GEN_DONE once its target length is reached); advance() takes the step's selection results."""
+
+    def __init__(self, P, policy=POLICY_SPECS, target_len=1024, sticky=False, p_target=0.5, max_steps=1 << 30):
+        self.P, self.policy, self.target_len, self.sticky = P, policy, int(target_len), bool(sticky)
+        self.p_target, self.max_steps = float(np.float32(p_target)), int(max_steps)
+        start = GEN_DRAFT if policy in (POLICY_ONLY_DRAFT, POLICY_DRAFT_START, POLICY_RSD) else GEN_TARGET
+        self.gen = [start] * P
+        self.length = [0] * P
+        self.steps = [0] * P
+        self.target_steps = [0] * P          # blocks appended that the target generated
+        self.target_calls = [0] * P          # generation rounds run by the target (RSD++ retries count)
+
+    def generators(self):
+        return [GEN_DONE if self._done(p) else self.gen[p] for p in range(self.P)]
+
+    def _done(self, p):
+        return self.length[p] >= self.target_len or self.steps[p] >= self.max_steps
+
+    def advance(self, chosen, flag, chosen_len, uniforms=None):
+        for p in range(self.P):
+            if self._done(p):
+                continue
+            g = self.gen[p]
+            if g == GEN_TARGET:
+                self.target_calls[p] += 1
+            if self.policy == POLICY_RSD and g == GEN_DRAFT and flag[p]:
+                self.gen[p] = GEN_TARGET          # the draft's best candidate is too weak: redo with the target
+                continue
+            if chosen[p] >= 0:
+                self.length[p] += int(chosen_len[p])
+                self.steps[p] += 1
+                if g == GEN_TARGET:
+                    self.target_steps[p] += 1
+            if self.policy == POLICY_SPECS:
+                if flag[p]:
+                    self.gen[p] = GEN_DRAFT
+                elif not self.sticky:
+                    self.gen[p] = GEN_TARGET
+            elif self.policy == POLICY_DRAFT_START:
+                if flag[p]:
+                    self.gen[p] = GEN_TARGET
+                elif not self.sticky:
+                    self.gen[p] = GEN_DRAFT
+            elif self.policy == POLICY_RANDOM:
+                self.gen[p] = GEN_TARGET if float(np.float32(uniforms[p])) < self.p_target else GEN_DRAFT
+            elif self.policy == POLICY_RSD:
+                self.gen[p] = GEN_DRAFT

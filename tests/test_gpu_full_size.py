@@ -71,6 +71,20 @@ def test_step7b_all_rows_all_betas(ctx, engine):
         got = s.step(cfg.betas[0], 0.7)
     finally:
         ctx.set_engine(binding.ENGINE_TCGEN05)
+    # the fused two-launch step, which is what bench.py times, gives the same bits as the separate calls
+    f = DeviceStep(ctx, x)
+    ctx.set_engine(engine)
+    try:
+        ctx.specs_beam_step(f.hidden, f.w_vocab, f.token_ids, f.block_offsets, f.cand_offsets, f.draft, f.reward,
+                            f.uniforms, cfg.betas[0], 0.7, f.tok_lp, f.blk_lp64, f.gen_blk64, f.weights, f.chosen,
+                            f.accept, f.workspace)
+        torch.cuda.synchronize()
+    finally:
+        ctx.set_engine(binding.ENGINE_TCGEN05)
+    fused = f.results()
+    for key in ("tok_logprob", "blk_logprob_f64", "blk_logprob_gen", "weights", "chosen", "accept"):
+        assert np.array_equal(fused[key], got[key]), key
+    del f
     w64 = O.bf16_bits_to_f64(x.w_vocab)
     all_rows = np.arange(x.rows)
     want_tok, err = check_sampled_rows(x, got["tok_logprob"], all_rows, w64)
