@@ -173,6 +173,43 @@ int specs_subsample_f64(specs_ctx* ctx, const double* blk_lp_target, const doubl
                         const float* uniforms, int32_t* chosen, float* weights,
                         float tau, uint8_t* accept, void* cuda_stream);
 
+/* Selection with the variants the paper uses in its comparisons and ablations.
+ *
+ * select_rule
+ *   SPECS_SELECT_SUBSAMPLE    Algorithm 2: a draw with P(i* = i) proportional to
+ *                             exp(S_i) * 1(i in L), by Gumbel-max on `uniforms`.
+ *   SPECS_SELECT_BEST_REWARD  the candidate of L with the highest reward, lowest index on
+ *                             ties: the selection of the PRM-guided beam-search baselines
+ *                             and of RSD++ (Section 4.1, Baselines); `uniforms` may be NULL;
+ *                             weights are 1 for the pick and 0 elsewhere.
+ * score_flags
+ *   SPECS_SCORE_NO_LL         S_i = beta * reward[i] even when blk_lp_gen is given: the
+ *                             "SPECS (no LL)" ablation of Section 4.3.
+ * mask  uint8 [total candidates] or NULL: the set L of Algorithm 2 (non-zero = member).
+ *       Candidates outside L get weight 0 and are never picked; a problem with no member
+ *       (or no candidate) gives chosen = -1.
+ * switch_rule, evaluated on the rewards of ALL candidates of the problem (in L or not):
+ *   SPECS_SWITCH_ANY_ABOVE    flag = max_i reward[i] > tau: Algorithm 1, Step III (the draft
+ *                             model may generate next).
+ *   SPECS_SWITCH_NONE_ABOVE   flag = no reward exceeds tau: the "pi_draft start" variant of
+ *                             Section 4.3 (the target model generates next).
+ *   SPECS_SWITCH_CHOSEN_BELOW flag = reward of the PICKED candidate < tau: RSD++'s rule
+ *                             (Section 4.1: redo the step with the target model).
+ *   A problem without candidates raises no flag.  flag may be NULL.
+ * Block log-probabilities are doubles as in specs_subsample_f64; blk_lp_gen == NULL means
+ * pi_gen = pi_target. */
+#define SPECS_SELECT_SUBSAMPLE    0
+#define SPECS_SELECT_BEST_REWARD  1
+#define SPECS_SCORE_NO_LL         0x1
+#define SPECS_SWITCH_ANY_ABOVE    0
+#define SPECS_SWITCH_NONE_ABOVE   1
+#define SPECS_SWITCH_CHOSEN_BELOW 2
+int specs_select(specs_ctx* ctx, const double* blk_lp_target, const double* blk_lp_gen,
+                 const float* reward, const uint8_t* mask, const int32_t* cand_offsets, int32_t P,
+                 float beta, const float* uniforms, int select_rule, int score_flags,
+                 int switch_rule, float tau, int32_t* chosen, float* weights, uint8_t* flag,
+                 void* cuda_stream);
+
 /* The dynamic-switching test alone (Algorithm 1, Step III; Section 2.3):
  * accept[p] = 1 iff the largest reward among ALL candidates of problem p is
  * strictly above tau, i.e. the draft model may generate the next step.  The call
@@ -206,6 +243,62 @@ int specs_beam_step(specs_ctx* ctx, const void* hidden, const void* W_vocab, con
                     float* tok_logprob, double* blk_logprob_f64, double* gen_blk_logprob_f64,
                     float* weights, int32_t* chosen, uint8_t* accept,
                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Host-side controller of the SPECS loop (Algorithm 1): for P problems it keeps which
+ * model drafts the next n candidate blocks, appends the selected block, applies the
+ * dynamic switch (Step III; Section 2.3) and stops at the target length.  All
+ * pointers are HOST pointers; nothing here touches a GPU.  One step of the loop:
+ *   specs_controller_generators  -> the caller drafts n blocks per problem with that
+ *                                   model, scores them (specs_beam_step / specs_select)
+ *   specs_controller_advance     <- chosen index, switch flag and length of the chosen
+ *                                   block, per problem.
+ *
+ * policy (Section 4.1 baselines and Section 4.3 ablations in brackets)
+ *   SPECS_POLICY_SPECS        starts with the target; flag (SPECS_SWITCH_ANY_ABOVE) = 1
+ *                             gives the next step to the draft.  sticky = 0: the test is
+ *                             taken anew at every step (Section 2.3); sticky = 1: once the
+ *                             draft, always the draft (Algorithm 1 read literally).
+ *   SPECS_POLICY_ONLY_DRAFT   every step from the draft ["Only Small Gen", BS(S)].
+ *   SPECS_POLICY_ONLY_TARGET  every step from the target [BS(B)].
+ *   SPECS_POLICY_RANDOM       after every step the target is chosen with probability
+ *                             p_target from a caller-supplied uniform ["Random Switch"].
+ *   SPECS_POLICY_DRAFT_START  starts with the draft; flag (SPECS_SWITCH_NONE_ABOVE) = 1
+ *                             gives the next step to the target ["SPECS (pi_draft start)"].
+ *   SPECS_POLICY_RSD          drafts with the draft; flag (SPECS_SWITCH_CHOSEN_BELOW) = 1
+ *                             discards the step and has the target redo it, whose pick
+ *                             is then appended unconditionally [RSD++].
+ * A problem is finished (generator SPECS_GEN_DONE, later updates ignored) once its
+ * appended length reaches target_len or its appended steps reach max_steps.  A step
+ * whose chosen index is -1 appends nothing. */
+#define SPECS_GEN_TARGET   0
+#define SPECS_GEN_DRAFT    1
+#define SPECS_GEN_DONE   (-1)
+#define SPECS_POLICY_SPECS        0
+#define SPECS_POLICY_ONLY_DRAFT   1
+#define SPECS_POLICY_ONLY_TARGET  2
+#define SPECS_POLICY_RANDOM       3
+#define SPECS_POLICY_DRAFT_START  4
+#define SPECS_POLICY_RSD          5
+typedef struct specs_controller specs_controller;
+typedef struct specs_policy {
+    int32_t policy;       /* SPECS_POLICY_* */
+    int32_t sticky;       /* see SPECS_POLICY_SPECS / SPECS_POLICY_DRAFT_START */
+    int64_t target_len;   /* tokens to append per problem */
+    int64_t max_steps;    /* blocks to append per problem at most */
+    float   p_target;     /* SPECS_POLICY_RANDOM: probability that the target generates, in [0, 1] */
+} specs_policy;
+int specs_controller_create(specs_controller** out, int32_t P, const specs_policy* policy);
+int specs_controller_destroy(specs_controller* ctrl);
+/* h_gen int32 [P] out: SPECS_GEN_TARGET, SPECS_GEN_DRAFT or SPECS_GEN_DONE. */
+int specs_controller_generators(const specs_controller* ctrl, int32_t* h_gen);
+/* h_chosen int32 [P], h_flag uint8 [P], h_chosen_len int64 [P] (tokens of the chosen block;
+ * ignored where h_chosen < 0), h_uniforms float [P] (SPECS_POLICY_RANDOM only, else may be NULL). */
+int specs_controller_advance(specs_controller* ctrl, const int32_t* h_chosen, const uint8_t* h_flag,
+                             const int64_t* h_chosen_len, const float* h_uniforms);
+/* Per problem, each int64 [P] out and optional: appended tokens, appended blocks, appended
+ * blocks that the target generated, generation rounds the target ran (RSD++ retries count). */
+int specs_controller_stats(const specs_controller* ctrl, int64_t* h_length, int64_t* h_steps,
+                           int64_t* h_target_steps, int64_t* h_target_calls);
 
 /* Synchronise `cuda_stream`, return the device status word (a combination of
  * SPECS_DEV_* bits, 0 if clean) through *h_bits and clear it.  Returns

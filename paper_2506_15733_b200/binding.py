@@ -26,6 +26,11 @@ DEV_TIMEOUT = 0x1
 DEV_TOKEN_RANGE = 0x2
 DEV_ACCUM_RANGE = 0x4
 ACCUM_ADAPTIVE = -1
+SELECT_SUBSAMPLE, SELECT_BEST_REWARD = 0, 1
+SCORE_NO_LL = 0x1
+SWITCH_ANY_ABOVE, SWITCH_NONE_ABOVE, SWITCH_CHOSEN_BELOW = 0, 1, 2
+GEN_TARGET, GEN_DRAFT, GEN_DONE = 0, 1, -1
+POLICY_SPECS, POLICY_ONLY_DRAFT, POLICY_ONLY_TARGET, POLICY_RANDOM, POLICY_DRAFT_START, POLICY_RSD = range(6)
 
 _vp, _i32, _i64, _f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
 
@@ -44,6 +49,13 @@ SIGNATURES = {
     "specs_subsample": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _f32, _vp, _vp, _vp, _f32, _vp, _vp]),
     "specs_subsample_f64": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _f32, _vp, _vp, _vp, _f32, _vp, _vp]),
     "specs_accept": (C.c_int, [_vp, _vp, _vp, _i32, _f32, _vp, _vp]),
+    "specs_select": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _f32, _vp, C.c_int, C.c_int, C.c_int, _f32,
+                               _vp, _vp, _vp, _vp]),
+    "specs_controller_create": (C.c_int, [C.POINTER(_vp), _i32, _vp]),
+    "specs_controller_destroy": (C.c_int, [_vp]),
+    "specs_controller_generators": (C.c_int, [_vp, _vp]),
+    "specs_controller_advance": (C.c_int, [_vp, _vp, _vp, _vp, _vp]),
+    "specs_controller_stats": (C.c_int, [_vp, _vp, _vp, _vp, _vp]),
     "specs_beam_step": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _f32, _f32,
                                   _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_size_t, _vp]),
     "specs_device_status": (C.c_int, [_vp, C.POINTER(C.c_uint32), _vp]),
@@ -204,6 +216,15 @@ class Context:
         _check(self._lib.specs_accept(self._h, _ptr(reward), _ptr(cand_offsets), P, float(tau), _ptr(accept),
                                       _stream()), "specs_accept")
 
+    def specs_select(self, blk_lp_target, blk_lp_gen, reward, mask, cand_offsets, beta, uniforms, select_rule,
+                     score_flags, switch_rule, tau, chosen, weights=None, flag=None):
+        """Selection with the paper's variants; block log-probabilities are float64 tensors."""
+        P = cand_offsets.shape[0] - 1
+        _check(self._lib.specs_select(self._h, _ptr(blk_lp_target), _ptr(blk_lp_gen), _ptr(reward), _ptr(mask),
+                                      _ptr(cand_offsets), P, float(beta), _ptr(uniforms), int(select_rule),
+                                      int(score_flags), int(switch_rule), float(tau), _ptr(chosen), _ptr(weights),
+                                      _ptr(flag), _stream()), "specs_select")
+
     def specs_beam_step(self, hidden, w_vocab, token_ids, block_offsets, cand_offsets, gen_tok_logprob, reward,
                         uniforms, beta, tau, tok_logprob, blk_logprob_f64, gen_blk_logprob_f64, weights, chosen,
                         accept, workspace):
@@ -232,6 +253,52 @@ class Context:
             _ptr(h_gen_tok_logprob), _ptr(h_reward), _ptr(h_uniforms), rows, d, V, B, P, float(beta), float(tau),
             _ptr(h_tok_logprob), _ptr(h_blk_logprob), _ptr(h_weights), _ptr(h_chosen), _ptr(h_accept), _stream()),
             "specs_beam_step_host")
+
+
+class Policy(C.Structure):
+    """Mirror of ``specs_policy``."""
+    _fields_ = [("policy", _i32), ("sticky", _i32), ("target_len", _i64), ("max_steps", _i64), ("p_target", _f32)]
+
+
+class Controller:
+    """Owns a ``specs_controller`` (host-side Algorithm 1 state for P problems); numpy arrays in and out."""
+
+    def __init__(self, P: int, policy: int = POLICY_SPECS, target_len: int = 1024, sticky: bool = False,
+                 p_target: float = 0.5, max_steps: int = 1 << 30):
+        self._lib = load_library()
+        self.P = int(P)
+        pol = Policy(int(policy), int(bool(sticky)), int(target_len), int(max_steps), float(p_target))
+        h = _vp()
+        _check(self._lib.specs_controller_create(C.byref(h), self.P, C.cast(C.byref(pol), _vp)),
+               "specs_controller_create")
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.specs_controller_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        self.close()
+
+    def generators(self) -> np.ndarray:
+        out = np.empty(self.P, np.int32)
+        _check(self._lib.specs_controller_generators(self._h, _ptr(out)), "specs_controller_generators")
+        return out
+
+    def advance(self, chosen, flag, chosen_len, uniforms=None):
+        chosen = np.ascontiguousarray(chosen, np.int32)
+        flag = np.ascontiguousarray(flag, np.uint8)
+        chosen_len = np.ascontiguousarray(chosen_len, np.int64)
+        uniforms = None if uniforms is None else np.ascontiguousarray(uniforms, np.float32)
+        _check(self._lib.specs_controller_advance(self._h, _ptr(chosen), _ptr(flag), _ptr(chosen_len),
+                                                  _ptr(uniforms)), "specs_controller_advance")
+
+    def stats(self) -> dict:
+        out = {k: np.empty(self.P, np.int64) for k in ("length", "steps", "target_steps", "target_calls")}
+        _check(self._lib.specs_controller_stats(self._h, *[_ptr(v) for v in out.values()]),
+               "specs_controller_stats")
+        return out
 
 
 NOALLOC_SCRATCH_BYTES = 8 << 20

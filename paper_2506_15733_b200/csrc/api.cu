@@ -336,6 +336,25 @@ int specs_subsample_f64(specs_ctx* ctx, const double* blk_lp_target, const doubl
                             weights, tau, accept, cuda_stream);
 }
 
+int specs_select(specs_ctx* ctx, const double* blk_lp_target, const double* blk_lp_gen, const float* reward,
+                 const uint8_t* mask, const int32_t* cand_offsets, int32_t P, float beta, const float* uniforms,
+                 int select_rule, int score_flags, int switch_rule, float tau, int32_t* chosen, float* weights,
+                 uint8_t* flag, void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    if (P < 0) return SPECS_ERR_SHAPE;
+    if (select_rule != SPECS_SELECT_SUBSAMPLE && select_rule != SPECS_SELECT_BEST_REWARD) return SPECS_ERR_SHAPE;
+    if (switch_rule < SPECS_SWITCH_ANY_ABOVE || switch_rule > SPECS_SWITCH_CHOSEN_BELOW) return SPECS_ERR_SHAPE;
+    if (score_flags & ~SPECS_SCORE_NO_LL) return SPECS_ERR_SHAPE;
+    if (P == 0) return SPECS_OK;
+    if (!reward || !cand_offsets || !chosen) return SPECS_ERR_NULL;
+    if (select_rule == SPECS_SELECT_SUBSAMPLE && !uniforms) return SPECS_ERR_NULL;
+    if (blk_lp_gen && !blk_lp_target) return SPECS_ERR_NULL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+    return launch_select(blk_lp_target, blk_lp_gen, reward, mask, cand_offsets, P, beta, uniforms, select_rule,
+                         score_flags, switch_rule, tau, chosen, weights, flag, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int specs_accept(specs_ctx* ctx, const float* reward, const int32_t* cand_offsets, int32_t P, float tau,
                  uint8_t* accept, void* cuda_stream) {
     if (!ctx) return SPECS_ERR_NULL;

@@ -175,6 +175,78 @@ __global__ void subsample_kernel(const LP* __restrict__ lp_t, const LP* __restri
                           weights, tau, accept);
 }
 
+// ------------------------------------------------------------------------------------ selection variants
+// Algorithm 2 with its candidate set L explicit (mask), the "highest reward" rule of the beam-search
+// and RSD++ baselines, the score without the log-ratio, and the three switch rules.  One warp per
+// problem; scores in double like subsample_problem.
+__global__ void select_kernel(const double* __restrict__ lp_t, const double* __restrict__ lp_g,
+                              const float* __restrict__ reward, const uint8_t* __restrict__ mask,
+                              const int32_t* __restrict__ cand_offsets, int32_t P, float beta,
+                              const float* __restrict__ uniforms, int select_rule, int score_flags,
+                              int switch_rule, float tau, int32_t* __restrict__ chosen,
+                              float* __restrict__ weights, uint8_t* __restrict__ flag) {
+    const int p = (int)(((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+    const int lane = threadIdx.x & 31;
+    if (p >= P) return;
+    const int a = cand_offsets[p], b = cand_offsets[p + 1];
+    const double* lq = (score_flags & SPECS_SCORE_NO_LL) ? nullptr : lp_g;
+    double smax = -INFINITY, best = -INFINITY;
+    int best_i = 0x7fffffff;
+    float rmax = -INFINITY;
+    for (int i = a + lane; i < b; i += 32) {
+        rmax = fmaxf(rmax, reward[i]);                       // the switch test sees every candidate
+        if (mask && mask[i] == 0) continue;
+        const double s = score_of(lp_t, lq, reward, beta, i);
+        smax = fmax(smax, s);
+        double key;
+        if (select_rule == SPECS_SELECT_BEST_REWARD) {
+            key = (double)reward[i];
+        } else {
+            float u = uniforms[i];
+            u = fminf(fmaxf(u, 2.98023223876953125e-8f), 0.99999994039535522461f);
+            key = s - log(-log((double)u));
+        }
+        if (key > best || best_i == 0x7fffffff) { best = key; best_i = i; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        smax = fmax(smax, __shfl_xor_sync(kFull, smax, o));
+        rmax = fmaxf(rmax, __shfl_xor_sync(kFull, rmax, o));
+        const double ob = __shfl_xor_sync(kFull, best, o);
+        const int oi = __shfl_xor_sync(kFull, best_i, o);
+        if (oi != 0x7fffffff && (best_i == 0x7fffffff || ob > best || (ob == best && oi < best_i))) {
+            best = ob; best_i = oi;
+        }
+    }
+    const bool none = best_i == 0x7fffffff;                  // empty problem, or nobody in L
+    if (weights) {
+        if (select_rule == SPECS_SELECT_BEST_REWARD || none) {
+            for (int i = a + lane; i < b; i += 32) weights[i] = (i == best_i) ? 1.0f : 0.0f;
+        } else {
+            double z = 0.0;
+            for (int i = a + lane; i < b; i += 32)
+                if (!mask || mask[i]) z += exp(score_of(lp_t, lq, reward, beta, i) - smax);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(kFull, z, o);
+            const double lse = smax + log(z);
+            for (int i = a + lane; i < b; i += 32)
+                weights[i] = (!mask || mask[i]) ? (float)exp(score_of(lp_t, lq, reward, beta, i) - lse) : 0.0f;
+        }
+    }
+    if (lane == 0) {
+        chosen[p] = none ? -1 : best_i - a;
+        if (flag) {
+            uint8_t f = 0;
+            if (b > a) {
+                if (switch_rule == SPECS_SWITCH_ANY_ABOVE) f = rmax > tau;
+                else if (switch_rule == SPECS_SWITCH_NONE_ABOVE) f = !(rmax > tau);
+                else f = !none && reward[best_i] < tau;
+            }
+            flag[p] = f;
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------ fused finish
 // Everything after the LM-head pass for one problem per CTA: merge the vocabulary splits of the
 // problem's rows, sum target and generator log-probabilities per drafted block, then SubSample and
@@ -294,6 +366,18 @@ int launch_subsample(const void* lp_target, const void* lp_gen, bool lp_is_f64, 
         subsample_kernel<float><<<blocks, threads, 0, stream>>>(
             static_cast<const float*>(lp_target), static_cast<const float*>(lp_gen), reward, cand_offsets, P, beta,
             uniforms, chosen, weights, tau, accept);
+    return cuda_status(cudaGetLastError());
+}
+
+int launch_select(const double* lp_target, const double* lp_gen, const float* reward, const uint8_t* mask,
+                  const int32_t* cand_offsets, int32_t P, float beta, const float* uniforms, int select_rule,
+                  int score_flags, int switch_rule, float tau, int32_t* chosen, float* weights, uint8_t* flag,
+                  cudaStream_t stream) {
+    if (P == 0) return SPECS_OK;
+    const int threads = 128;
+    select_kernel<<<warps_grid(P, threads), threads, 0, stream>>>(lp_target, lp_gen, reward, mask, cand_offsets, P,
+                                                                   beta, uniforms, select_rule, score_flags,
+                                                                   switch_rule, tau, chosen, weights, flag);
     return cuda_status(cudaGetLastError());
 }
 

@@ -128,6 +128,10 @@ int launch_block_sums(const float* per_token, const int64_t* block_offsets, int3
 int launch_subsample(const void* lp_target, const void* lp_gen, bool lp_is_f64, const float* reward,
                      const int32_t* cand_offsets, int32_t P, float beta, const float* uniforms,
                      int32_t* chosen, float* weights, float tau, uint8_t* accept, cudaStream_t stream);
+int launch_select(const double* lp_target, const double* lp_gen, const float* reward, const uint8_t* mask,
+                  const int32_t* cand_offsets, int32_t P, float beta, const float* uniforms, int select_rule,
+                  int score_flags, int switch_rule, float tau, int32_t* chosen, float* weights, uint8_t* flag,
+                  cudaStream_t stream);
 int launch_accept(const float* reward, const int32_t* cand_offsets, int32_t P, float tau,
                   uint8_t* accept, cudaStream_t stream);
 

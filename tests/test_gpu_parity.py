@@ -438,3 +438,112 @@ def test_adaptive_chunks_flag_logits_beyond_the_sampled_magnitude(ctx):
         ctx.set_accum_chunk(binding.ACCUM_ADAPTIVE)
     assert ctx.device_status() == 0
     assert np.abs(got - want).max() <= TOK_ATOL
+
+
+# ------------------------------------------------------------------------------- selection variants
+
+from oracle import specs_variants as OV   # noqa: E402
+
+
+@pytest.mark.parametrize("select_rule", [OV.SELECT_SUBSAMPLE, OV.SELECT_BEST_REWARD])
+@pytest.mark.parametrize("score_flags", [0, OV.SCORE_NO_LL])
+@pytest.mark.parametrize("masked", [False, True])
+def test_select_variants_match_the_oracle(ctx, select_rule, score_flags, masked):
+    rng = np.random.Generator(np.random.Philox(key=[5400, select_rule * 4 + score_flags * 2 + masked]))
+    sizes = rng.integers(0, 70, size=1500)
+    cand = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    B, P = int(cand[-1]), len(sizes)
+    lp_t = rng.uniform(-4000, -5, B)
+    lp_g = lp_t + rng.normal(0, 3.0, B)
+    r = rng.random(B).astype(np.float32)
+    r[rng.integers(0, B, 200)] = np.float32(0.5)                    # ties in the reward
+    u = I.draw_uniforms(5401, B)
+    mask = (rng.random(B) < 0.6).astype(np.uint8) if masked else None
+    if masked:
+        mask[cand[10]:cand[11]] = 0                                 # a problem with nobody in L
+    dev = "cuda:0"
+    t = lambda a: None if a is None else torch.from_numpy(a).to(dev)
+    d_in = [t(lp_t), t(lp_g), t(r), t(mask), t(cand)]
+    chosen = torch.full((P,), -7, dtype=torch.int32, device=dev)
+    wts = torch.full((B,), float("nan"), dtype=torch.float32, device=dev)
+    flag = torch.full((P,), 9, dtype=torch.uint8, device=dev)
+    want_c, want_w, margin = OV.select(lp_t, lp_g, r, mask, cand, 2.0, u, select_rule, score_flags)
+    for switch_rule in (OV.SWITCH_ANY_ABOVE, OV.SWITCH_NONE_ABOVE, OV.SWITCH_CHOSEN_BELOW):
+        ctx.specs_select(*d_in, 2.0, t(u), select_rule, score_flags, switch_rule, 0.8, chosen, wts, flag)
+        torch.cuda.synchronize()
+        got_c = chosen.cpu().numpy()
+        sure = (margin > MARGIN) | (select_rule == OV.SELECT_BEST_REWARD)   # the reward comparison is exact
+        assert np.array_equal(got_c[sure], want_c[sure])
+        assert np.array_equal(got_c == -1, want_c == -1)
+        assert np.abs(wts.cpu().numpy() - want_w).max() < 1e-6
+        # flags follow the oracle given the GPU's own pick (they coincide wherever the pick is sure)
+        assert np.array_equal(flag.cpu().numpy(), OV.switch_flags(r, cand, got_c, 0.8, switch_rule))
+    if masked:
+        picked = cand[:-1][got_c >= 0] + got_c[got_c >= 0]
+        assert mask[picked].all() and got_c[10] == -1
+
+
+def test_select_rejects_unknown_rules(ctx):
+    dev = "cuda:0"
+    r = torch.zeros(4, dtype=torch.float32, device=dev)
+    cand = torch.tensor([0, 4], dtype=torch.int32, device=dev)
+    chosen = torch.zeros(1, dtype=torch.int32, device=dev)
+    for args in ((2, 0, 0), (0, 2, 0), (0, 0, 3)):
+        with pytest.raises(binding.SpecsError) as e:
+            ctx.specs_select(None, None, r, None, cand, 1.0, r, args[0], args[1], args[2], 0.5, chosen)
+        assert e.value.status == 2
+    with pytest.raises(binding.SpecsError) as e:
+        ctx.specs_select(None, None, r, None, cand, 1.0, None, OV.SELECT_SUBSAMPLE, 0, 0, 0.5, chosen)
+    assert e.value.status == 1                                      # Algorithm 2 needs its uniforms
+    ctx.specs_select(None, None, r, None, cand, 1.0, None, OV.SELECT_BEST_REWARD, 0, 0, 0.5, chosen)
+    torch.cuda.synchronize()
+    assert chosen.item() == 0                                       # all rewards equal: lowest index
+
+
+def test_specs_loop_with_stub_generators(ctx):
+    # Algorithm 1 end to end for a few steps: the native controller decides who drafts, stub generators
+    # (seeded random blocks and hidden states, a higher reward level for the target's blocks) stand in
+    # for the models, the CUDA path scores and selects; the oracle runs the same loop on the CPU.
+    P, n, d, Vv = 3, 4, 64, 500
+    got_ctl = binding.Controller(P, binding.POLICY_SPECS, target_len=60)
+    want_ctl = OV.Controller(P, OV.POLICY_SPECS, target_len=60)
+    w_cfg = small_config("loop_w", (1, 1), 1, 1, d, Vv, seed=5500)
+    w_bits = I.make_step_inputs(w_cfg).w_vocab
+    trace_got, trace_want = [], []
+    for step in range(8):
+        gens = got_ctl.generators()
+        assert gens.tolist() == want_ctl.generators()
+        live = [p for p in range(P) if gens[p] != binding.GEN_DONE]
+        if not live:
+            break
+        cfg = small_config("loop", (4, 12), len(live), n, d, Vv, seed=5510 + step)
+        x = I.make_step_inputs(cfg)
+        x.w_vocab = w_bits                                          # the same LM head at every step
+        for j, p in enumerate(live):                                # the target's candidates score higher
+            if gens[p] == binding.GEN_TARGET:
+                x.reward[j * n:(j + 1) * n] = np.float32(0.5) + x.reward[j * n:(j + 1) * n] / 2
+            else:
+                x.reward[j * n:(j + 1) * n] /= 2
+        s = DeviceStep(ctx, x)
+        ctx.specs_beam_step(s.hidden, s.w_vocab, s.token_ids, s.block_offsets, s.cand_offsets, s.draft, s.reward,
+                            s.uniforms, 1.0, 0.8, s.tok_lp, s.blk_lp64, s.gen_blk64, s.weights, s.chosen, s.accept,
+                            s.workspace)
+        torch.cuda.synchronize()
+        g = s.results()
+        ref = oracle_step(x, 1.0, 0.8)
+        lens = np.diff(x.block_offsets)
+        for ctl, res, trace in ((got_ctl, g, trace_got), (want_ctl, ref, trace_want)):
+            chosen = np.full(P, -1, np.int32); flag = np.zeros(P, np.uint8); clen = np.zeros(P, np.int64)
+            for j, p in enumerate(live):
+                chosen[p] = res["chosen"][j]; flag[p] = res["accept"][j]
+                clen[p] = lens[j * n + res["chosen"][j]]
+            ctl.advance(chosen, flag, clen)
+            trace.append((chosen.tolist(), flag.tolist()))
+        if np.all(ref["margin"] > MARGIN + 1e-2):
+            assert trace_got[-1] == trace_want[-1]
+        else:                                                       # an unsure pick: keep both loops on one path
+            want_ctl.length, want_ctl.steps = got_ctl.stats()["length"].tolist(), got_ctl.stats()["steps"].tolist()
+            want_ctl.target_steps = got_ctl.stats()["target_steps"].tolist()
+    st = got_ctl.stats()
+    assert st["steps"].sum() >= P and (st["target_steps"] >= 1).all()   # every problem began with the target
+    assert ctx.device_status() == 0
