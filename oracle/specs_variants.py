@@ -150,3 +150,42 @@ class Controller:
                 self.gen[p] = GEN_TARGET if float(np.float32(uniforms[p])) < self.p_target else GEN_DRAFT
             elif self.policy == POLICY_RSD:
                 self.gen[p] = GEN_DRAFT
+
+
+# --------------------------------------------------------------------------- both heads, and the append
+
+def beam_step_dual(hidden_target_bits, w_target_bits, hidden_gen_bits, w_gen_bits, token_ids, block_offsets,
+                   cand_offsets, reward, beta, uniforms, tau):
+    """The step when the generator's log-probabilities are not given but computed: the drafted tokens are
+    scored with the generator's own LM head (its hidden states and weights) exactly as with the target's
+    (Section 2; the latency breakdown of Appendix E.1 lists scoring with the draft and with the target),
+    and Eq. (1) takes the two block log-probabilities."""
+    from oracle import specs_oracle as O
+    lp_t = O.token_logprobs(hidden_target_bits, w_target_bits, token_ids)
+    lp_g = O.token_logprobs(hidden_gen_bits, w_gen_bits, token_ids)
+    LP, LQ = O.block_sums(lp_t, block_offsets), O.block_sums(lp_g, block_offsets)
+    S = O.scores(LP, LQ, reward, beta)
+    chosen, margin = O.gumbel_pick(S, uniforms, cand_offsets)
+    return {"tok_logprob": lp_t, "gen_tok_logprob": lp_g, "tok_logratio": lp_t - lp_g, "blk_logprob": LP,
+            "blk_logprob_gen": LQ, "score": S, "weights": O.weights(S, cand_offsets), "chosen": chosen,
+            "margin": margin, "accept": O.accept_flags(reward, cand_offsets, tau)}
+
+
+def gather_chosen(token_ids, block_offsets, cand_offsets, chosen, stride):
+    """Step II of Algorithm 1 appends the selected block to the trace: the ids of block
+    (first block of the problem + chosen) go to row p of an int32 [P, stride] array (-1 beyond the block's
+    length, everything -1 when nothing was chosen), its length to chosen_len[p]."""
+    P = len(cand_offsets) - 1
+    out = np.full((P, stride), -1, dtype=np.int32)
+    lens = np.zeros(P, dtype=np.int32)
+    for p in range(P):
+        if chosen[p] < 0:
+            continue
+        blk = int(cand_offsets[p]) + int(chosen[p])
+        a, b = int(block_offsets[blk]), int(block_offsets[blk + 1])
+        if b - a > stride:
+            raise ValueError("chosen block longer than the output row")
+        for k in range(a, b):
+            out[p, k - a] = token_ids[k]
+        lens[p] = b - a
+    return out, lens

@@ -168,3 +168,48 @@ def test_random_switching_matches_the_requested_share_of_target_steps():
     share = np.mean(np.array(seen[1:]) == V.GEN_TARGET)
     assert abs(share - p) < 4 * np.sqrt(p * (1 - p) / steps)
     assert c.target_steps[0] == sum(g == V.GEN_TARGET for g in seen[:-1])
+
+
+# ------------------------------------------------------------------------------- both heads, and the append
+
+def test_dual_step_is_eq_1_with_both_block_probabilities_computed():
+    # tiny case by brute force: every probability from explicit softmaxes in Python floats
+    import math
+    rng = np.random.Generator(np.random.Philox(key=[6800, 1]))
+    Vv, rows = 5, 6
+    def bits(a):
+        return (np.asarray(a, np.float32).view(np.uint32) >> 16).astype(np.uint16)       # values exact in bf16
+    Ht = bits(rng.integers(-4, 5, (rows, 8)) / 4.0); Wt = bits(rng.integers(-4, 5, (Vv, 8)) / 8.0)
+    Hg = bits(rng.integers(-4, 5, (rows, 16)) / 4.0); Wg = bits(rng.integers(-4, 5, (Vv, 16)) / 8.0)
+    ids = rng.integers(0, Vv, rows).astype(np.int32)
+    boff = np.array([0, 2, 3, 6]); cand = np.array([0, 3])
+    r = np.array([0.3, 0.8, 0.5], np.float32); u = np.array([0.2, 0.5, 0.7], np.float32)
+    got = V.beam_step_dual(Ht, Wt, Hg, Wg, ids, boff, cand, r, 2.0, u, 0.7)
+
+    def lp(H, W, t):
+        h = O.bf16_bits_to_f64(H)[t].tolist(); w = O.bf16_bits_to_f64(W).tolist()
+        z = [sum(a * b for a, b in zip(h, wv)) for wv in w]
+        return z[ids[t]] - math.log(sum(math.exp(v) for v in z))
+    S = []
+    for i in range(3):
+        ratio = sum(lp(Ht, Wt, t) - lp(Hg, Wg, t) for t in range(boff[i], boff[i + 1]))
+        S.append(ratio + 2.0 * float(r[i]))
+    assert np.allclose(got["score"], S, rtol=1e-12)
+    assert np.allclose(got["tok_logratio"].sum(), sum(S) - 2.0 * float(r.sum()), rtol=1e-12)
+    pert = [S[i] - math.log(-math.log(float(u[i]))) for i in range(3)]
+    assert got["chosen"][0] == pert.index(max(pert)) and got["accept"][0] == 1
+    # identical heads: the ratio vanishes and the score collapses to beta * r (text after Eq. 1)
+    same = V.beam_step_dual(Ht, Wt, Ht, Wt, ids, boff, cand, r, 2.0, u, 0.7)
+    assert np.allclose(same["score"], 2.0 * r.astype(np.float64), atol=1e-12)
+
+
+def test_gather_chosen_worked_example():
+    ids = np.arange(100, 112, dtype=np.int32)
+    boff = np.array([0, 3, 3, 7, 9, 12]); cand = np.array([0, 2, 2, 5])
+    out, lens = V.gather_chosen(ids, boff, cand, np.array([0, -1, 2]), 4)
+    assert out.tolist() == [[100, 101, 102, -1], [-1, -1, -1, -1], [109, 110, 111, -1]]
+    assert lens.tolist() == [3, 0, 3]
+    out, lens = V.gather_chosen(ids, boff, cand, np.array([1, -1, 0]), 4)       # an empty block is a valid pick
+    assert out[0].tolist() == [-1] * 4 and lens.tolist() == [0, 0, 4] and out[2].tolist() == [103, 104, 105, 106]
+    with pytest.raises(ValueError):
+        V.gather_chosen(ids, boff, cand, np.array([0, -1, 0]), 3)
