@@ -172,6 +172,8 @@ def main():
     ap.add_argument("--config", default="step7b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--oracle-blocks", type=int, default=16, help="whole blocks per CPU-oracle sample")
+    ap.add_argument("--tile-lead", type=int, default=None,
+                    help="pacing of the CTA pairs that stream the same W chunk, in vocabulary tiles (0: off; default: the library's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -206,6 +208,8 @@ def main():
     rows, B, P, d, V = x.rows, x.blocks, cfg.problems, cfg.d, cfg.vocab
     beta, tau = cfg.betas[0], cfg.taus[0]
     ctx = binding.Context(local_rank)
+    if args.tile_lead is not None:
+        ctx.set_tile_lead(args.tile_lead)
 
     # device-resident copies
     t = lambda a: torch.from_numpy(a).to(dev)

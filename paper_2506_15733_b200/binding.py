@@ -41,6 +41,7 @@ SIGNATURES = {
     "specs_destroy": (C.c_int, [_vp]),
     "specs_set_engine": (C.c_int, [_vp, C.c_int]),
     "specs_set_accum_chunk": (C.c_int, [_vp, _i32]),
+    "specs_set_tile_lead": (C.c_int, [_vp, _i32]),
     "specs_sm_count": (C.c_int, [_vp]),
     "specs_score_workspace_bytes": (C.c_size_t, [_vp, _i64, _i32, _i32]),
     "specs_score_blocks": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp,
@@ -160,6 +161,9 @@ class Context:
 
     def set_accum_chunk(self, k_elements: int):
         _check(self._lib.specs_set_accum_chunk(self._h, int(k_elements)), "specs_set_accum_chunk")
+
+    def set_tile_lead(self, tiles: int):
+        _check(self._lib.specs_set_tile_lead(self._h, int(tiles)), "specs_set_tile_lead")
 
     def sm_count(self) -> int:
         return int(self._lib.specs_sm_count(self._h))

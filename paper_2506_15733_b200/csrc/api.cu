@@ -86,8 +86,7 @@ ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, i
 }
 
 size_t plan_workspace_bytes(const ScorePlan& p) {
-    const size_t slots = (size_t)(p.waves > 0 ? p.waves : 1) * (size_t)p.grid;
-    return slots * kTripleFloats * sizeof(float);
+    return plan_slot_bytes(p) + (size_t)p.units * sizeof(uint64_t);
 }
 
 }  // namespace specs
@@ -217,6 +216,13 @@ int specs_set_accum_chunk(specs_ctx* ctx, int32_t k_elements) {
     if (k_elements < 0 || (k_elements % kBlockK) != 0) return SPECS_ERR_SHAPE;
     ctx->chunk_kblocks = k_elements / kBlockK;               // 0: one accumulator over the whole of d
     ctx->accum_adaptive = false;
+    return SPECS_OK;
+}
+
+int specs_set_tile_lead(specs_ctx* ctx, int32_t tiles) {
+    if (!ctx) return SPECS_ERR_NULL;
+    if (tiles < 0 || tiles > 1024) return SPECS_ERR_SHAPE;
+    ctx->lead_tiles = tiles;
     return SPECS_OK;
 }
 

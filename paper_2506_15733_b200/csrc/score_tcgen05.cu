@@ -51,7 +51,13 @@
 // kernel returns.
 #include <cuda_bf16.h>
 
+#include <atomic>
+
 #include "specs_internal.h"
+
+#ifndef SPECS_TMA_HINTS
+#define SPECS_TMA_HINTS 0
+#endif
 
 namespace specs {
 namespace {
@@ -199,6 +205,33 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c_inner), "r"(c_outer), "r"(cluster_bar)
         : "memory");
 }
+// L2 eviction-priority policies for the two operand streams.
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer,
+                                                 uint32_t bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c_inner), "r"(c_outer), "r"(bar), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair_hint(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer,
+                                                      uint32_t cluster_bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c_inner), "r"(c_outer), "r"(cluster_bar), "l"(policy)
+        : "memory");
+}
 // 2^x on the special-function unit (relative error about 2^-22; 2^-inf = 0).
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
@@ -283,6 +316,28 @@ __device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t saddr) {
 __host__ __device__ constexpr uint32_t instr_desc_bf16(int m, int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
            (static_cast<uint32_t>(m >> 4) << 24);
+}
+
+// ---- pacing of the units that stream the same W chunk ------------------------------------------
+// Units that share a vocabulary chunk read the same W tiles; only while they stay within a few
+// tiles of each other does each tile come from HBM once and from L2 for the rest.  Every unit's
+// producer publishes (epoch, wave, tile) when it starts a tile and, before starting tile t, waits
+// until no unit of its group is further back than t - lead.  The wait is advisory: it gives up
+// after a short time, and for good after a few expiries, so stale or foreign workspace contents
+// can only cost time.
+constexpr unsigned long long kPaceLimitNs = 40000ull;       // per tile
+constexpr int kPaceMaxExpiries = 4;
+__device__ __forceinline__ unsigned long long pace_key(uint32_t epoch, int wave, int tile) {
+    return ((unsigned long long)(epoch & 0xffffu) << 48) | ((unsigned long long)(wave & 0xffffff) << 24) |
+           (unsigned long long)(tile & 0xffffff);
+}
+__device__ __forceinline__ unsigned long long ld_progress(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_progress(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 
 struct SharedLayout {
@@ -390,17 +445,61 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kControlRegs));
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            // pair: every load of either CTA is counted on the leader's barrier of the stage
-            const uint32_t full0 = (kCg == 2) ? mapa_shared(smem_u32(&sh->full[0]), 0u) : smem_u32(&sh->full[0]);
-            uint32_t stage = 0, phase = 0;
-            uint32_t issued = 0;
-            bool ok = true;
-            for (int w = 0; w < plan.waves && ok; ++w) {
-                int st, nb, ne;
-                if (!plan_unit(plan, w, unit, &st, &nb, &ne)) continue;
-                const int row0 = (st * kCg + (int)rank) * kBlockM;
-                for (int n = nb; n < ne && ok; ++n) {
+        // Lane 0 waits for free stages and issues the loads; the whole warp takes part in the pacing
+        // poll before each vocabulary tile (one progress word per lane, one trip to L2).
+        // pair: every load of either CTA is counted on the leader's barrier of the stage
+        const uint32_t full0 = (kCg == 2) ? mapa_shared(smem_u32(&sh->full[0]), 0u) : smem_u32(&sh->full[0]);
+#if SPECS_TMA_HINTS == 1
+        const uint64_t pol_h = l2_policy_evict_last(), pol_w = l2_policy_evict_first();
+#elif SPECS_TMA_HINTS == 2
+        const uint64_t pol_h = l2_policy_evict_last(), pol_w = l2_policy_evict_last();
+#elif SPECS_TMA_HINTS == 3
+        const uint64_t pol_h = l2_policy_evict_first(), pol_w = l2_policy_evict_last();
+#endif
+        unsigned long long* progress = reinterpret_cast<unsigned long long*>(
+            reinterpret_cast<char*>(workspace) + plan_slot_bytes(plan));
+        bool pace = plan.lead_tiles > 0 && rank == 0;
+        int expiries = 0;
+        uint32_t stage = 0, phase = 0;           // meaningful in lane 0 only
+        uint32_t issued = 0;
+        bool ok = true;                          // warp-uniform
+        for (int w = 0; w < plan.waves && ok; ++w) {
+            int st, nb, ne;
+            if (!plan_unit(plan, w, unit, &st, &nb, &ne)) continue;
+            const int row0 = (st * kCg + (int)rank) * kBlockM;
+            // the units of this wave that stream the same vocabulary chunk
+            const int gm_w = w < plan.full_waves ? plan.group_m : plan.rem_m;
+            const int group0 = (unit / gm_w) * gm_w;
+            for (int n = nb; n < ne && ok; ++n) {
+                if (pace && gm_w > 1) {
+                    const int t = n - nb;
+                    if (lane == 0) st_progress(progress + unit, pace_key(plan.epoch, w, t));
+                    if (t >= plan.lead_tiles) {
+                        const unsigned long long need = pace_key(plan.epoch, w, t - plan.lead_tiles);
+                        const unsigned long long t0 = global_timer_ns();
+                        for (;;) {
+                            unsigned long long lo = ~0ull;
+                            for (int i = lane; i < gm_w; i += 32) {
+                                const unsigned long long v = ld_progress(progress + group0 + i);
+                                // a word of another launch counts as "not started"
+                                const unsigned long long cur = (v >> 48) == (plan.epoch & 0xffffu) ? v : 0ull;
+                                lo = cur < lo ? cur : lo;
+                            }
+#pragma unroll
+                            for (int o = 16; o > 0; o >>= 1) {
+                                const unsigned long long other = __shfl_xor_sync(0xffffffffu, lo, o);
+                                lo = other < lo ? other : lo;
+                            }
+                            const bool expired = __shfl_sync(0xffffffffu, global_timer_ns() - t0 > kPaceLimitNs, 0);
+                            if (lo >= need) { expiries = 0; break; }
+                            if (expired) {
+                                if (++expiries >= kPaceMaxExpiries) pace = false;
+                                break;
+                            }
+                        }
+                    }
+                }
+                if (lane == 0) {
                     const int wrow0 = n * kBlockN + (int)rank * S::kBRows;
                     for (int kb = 0; kb < plan.k_blocks; ++kb) {
                         if (!mbar_wait(smem_u32(&sh->empty[stage]), phase ^ 1u, ab, kWaitLimitNs, true)) {
@@ -408,23 +507,30 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                             break;
                         }
                         const uint32_t a_dst = tiles_addr + stage * kStageBytes;
+                        const uint32_t bar = full0 + stage * 8u;
                         if (kCg == 1) {
-                            const uint32_t bar = full0 + stage * 8u;
                             mbar_arrive_expect_tx(bar, kStageBytes);
                             tma_load_2d(a_dst, &map_hidden, kb * kBlockK, row0, bar);
                             tma_load_2d(a_dst + kABytes, &map_w, kb * kBlockK, wrow0, bar);
                         } else {
-                            const uint32_t bar = full0 + stage * 8u;
                             // the leader expects both CTAs' bytes; the peer's may be counted first
                             if (rank == 0) mbar_arrive_expect_tx(smem_u32(&sh->full[stage]), 2u * kStageBytes);
+#if SPECS_TMA_HINTS
+                            tma_load_2d_pair_hint(a_dst, &map_hidden, kb * kBlockK, row0, bar, pol_h);
+                            tma_load_2d_pair_hint(a_dst + kABytes, &map_w, kb * kBlockK, wrow0, bar, pol_w);
+#else
                             tma_load_2d_pair(a_dst, &map_hidden, kb * kBlockK, row0, bar);
                             tma_load_2d_pair(a_dst + kABytes, &map_w, kb * kBlockK, wrow0, bar);
+#endif
                         }
                         ++issued;
                         if (++stage == kStages) { stage = 0; phase ^= 1u; }
                     }
                 }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
             }
+        }
+        if (lane == 0) {
             if (ok) {
                 // Tail: wait until the MMAs that read the last stages have retired, so that no
                 // barrier arrival (in the pair kernel: from the other CTA) is still on its way
@@ -729,13 +835,17 @@ int query_pair_units(int device, int num_sms) {
     return units;
 }
 
-int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan, const void* hidden, const void* w_vocab,
+int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan_in, const void* hidden, const void* w_vocab,
                          const int32_t* token_ids, float* workspace, cudaStream_t stream) {
     static_assert(Shape<1>::kSmemBytes <= 227 * 1024 && Shape<2>::kSmemBytes <= 227 * 1024, "shared memory budget");
     static_assert(Shape<1>::kStages <= kMaxStages && Shape<2>::kStages <= kMaxStages, "barrier arrays");
     static_assert(sizeof(SharedLayout) <= 512, "barrier block");
-    const bool pair = plan.cta_group == 2;
-    if (pair && (plan.units > ctx->pair_units || (plan.grid & 1))) return SPECS_ERR_CUDA;
+    const bool pair = plan_in.cta_group == 2;
+    if (pair && (plan_in.units > ctx->pair_units || (plan_in.grid & 1))) return SPECS_ERR_CUDA;
+    static std::atomic<uint32_t> launch_counter{0};
+    ScorePlan plan = plan_in;
+    plan.epoch = (launch_counter.fetch_add(1) % 0xfffeu) + 1u;  // never 0
+    plan.lead_tiles = ctx->lead_tiles;
     query_pair_units(ctx->device, ctx->num_sms);             // shared-memory opt-in for this device
     CUtensorMap map_h, map_w;
     int st = encode_bf16_2d(ctx, &map_h, hidden, (uint64_t)plan.d, (uint64_t)plan.rows, kBlockK, kBlockM);

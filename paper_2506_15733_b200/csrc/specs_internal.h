@@ -51,6 +51,9 @@ struct ScorePlan {
     int32_t split_rem;     // vocab chunks of the last wave
     int32_t waves;         // full_waves + (rem_m > 0)
     int32_t chunk_kblocks; // k-blocks per fresh tensor-core accumulator (chunks are summed in registers)
+    int32_t lead_tiles;    // > 0: a unit starts vocabulary tile t of a wave only once every unit that streams the
+                           //      same W chunk has started tile t - lead_tiles (advisory, bounded wait)
+    uint32_t epoch;        // distinguishes this launch's progress words from older contents of the workspace
     int32_t adaptive;      // 1: from the third vocabulary tile of a run on, lengthen the chunks as far as the
                            //    logit magnitude seen in the run's first tile allows (see score_tcgen05.cu)
 };
@@ -64,6 +67,10 @@ ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, i
                           int32_t cta_group = kCtaGroupAuto, int32_t chunk_kblocks = kDefaultChunkKBlocks,
                           bool adaptive = true);
 size_t plan_workspace_bytes(const ScorePlan& p);
+// The workspace: triple slots [waves x grid], then one 64-bit progress word per unit.
+__host__ __device__ inline size_t plan_slot_bytes(const ScorePlan& p) {
+    return (size_t)(p.waves > 0 ? p.waves : 1) * (size_t)p.grid * kTripleFloats * sizeof(float);
+}
 
 // Work unit `unit` in wave `wave`: returns false when the unit idles in that wave.
 __host__ __device__ inline bool plan_unit(const ScorePlan& p, int wave, int unit,
@@ -95,6 +102,7 @@ struct specs_ctx {
     int pair_units = 0;                    // resident CTA pairs of the pair kernel (0: not available)
     int chunk_kblocks = specs::kDefaultChunkKBlocks;   // see specs_set_accum_chunk
     bool accum_adaptive = true;
+    int lead_tiles = 1;                    // see specs_set_tile_lead
     uint32_t* d_status = nullptr;          // device status word (SPECS_DEV_* bits)
     specs::EncodeTiledFn encode_tiled = nullptr;
     // grow-only device arena for specs_beam_step_host
