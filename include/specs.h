@@ -252,6 +252,42 @@ int specs_beam_step(specs_ctx* ctx, const void* hidden, const void* W_vocab, con
                     float* weights, int32_t* chosen, uint8_t* accept,
                     void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* The beam step when the generator's log-probabilities are computed rather than
+ * given: the drafted tokens are scored with the generator's own LM head as well
+ * (its final hidden states hidden_gen [rows, d_gen] and weights W_gen [V, d_gen];
+ * Appendix E.1 lists scoring with the draft and with the target model), and Eq. (1)
+ * takes the two block log-probabilities.  Three launches: the generator-shaped
+ * scoring pass, the target-shaped one, and one finish kernel that merges both,
+ * writes both per-token log-probabilities (their difference is the per-token
+ * log-ratio), sums them per block, runs SubSample and the switch test and, when
+ * chosen_ids is given, gathers the selected block's token ids for the append of
+ * Algorithm 1, Step II (see specs_gather_chosen).
+ *
+ *   gen_tok_logprob  float [rows] OUT here.  Both heads share the vocabulary size V.
+ *   chosen_ids       int32 [P, chosen_stride] out or NULL; chosen_len int32 [P] out.
+ *   workspace        at least specs_beam_step_dual_workspace_bytes().
+ * Everything else as in specs_beam_step. */
+size_t specs_beam_step_dual_workspace_bytes(const specs_ctx* ctx, int64_t rows, int32_t d_target,
+                                            int32_t d_gen, int32_t V);
+int specs_beam_step_dual(specs_ctx* ctx, const void* hidden_target, const void* W_target, int32_t d_target,
+                         const void* hidden_gen, const void* W_gen, int32_t d_gen,
+                         const int32_t* token_ids, const int64_t* block_offsets,
+                         const int32_t* cand_offsets, const float* reward, const float* uniforms,
+                         int64_t rows, int32_t V, int32_t B, int32_t P, float beta, float tau,
+                         float* tok_logprob, float* gen_tok_logprob, double* blk_logprob_f64,
+                         double* gen_blk_logprob_f64, float* weights, int32_t* chosen, uint8_t* accept,
+                         int32_t* chosen_ids, int32_t* chosen_len, int32_t chosen_stride,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* What Step II of Algorithm 1 appends to the trace: for every problem the token ids
+ * of its selected block (block cand_offsets[p] + chosen[p]) go to row p of
+ * chosen_ids [P, chosen_stride], padded with -1, and the block's length to
+ * chosen_len[p]; chosen[p] = -1 gives a row of -1 and length 0.  The caller makes
+ * chosen_stride at least the longest block (longer blocks are cut to the stride). */
+int specs_gather_chosen(specs_ctx* ctx, const int32_t* token_ids, const int64_t* block_offsets,
+                        const int32_t* cand_offsets, const int32_t* chosen, int32_t P,
+                        int32_t* chosen_ids, int32_t* chosen_len, int32_t chosen_stride, void* cuda_stream);
+
 /* Host-side controller of the SPECS loop (Algorithm 1): for P problems it keeps which
  * model drafts the next n candidate blocks, appends the selected block, applies the
  * dynamic switch (Step III; Section 2.3) and stops at the target length.  All

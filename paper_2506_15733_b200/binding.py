@@ -59,6 +59,11 @@ SIGNATURES = {
     "specs_controller_stats": (C.c_int, [_vp, _vp, _vp, _vp, _vp]),
     "specs_beam_step": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _f32, _f32,
                                   _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_size_t, _vp]),
+    "specs_beam_step_dual_workspace_bytes": (C.c_size_t, [_vp, _i64, _i32, _i32, _i32]),
+    "specs_beam_step_dual": (C.c_int, [_vp, _vp, _vp, _i32, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32,
+                                       _i32, _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp,
+                                       C.c_size_t, _vp]),
+    "specs_gather_chosen": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _i32, _vp]),
     "specs_device_status": (C.c_int, [_vp, C.POINTER(C.c_uint32), _vp]),
     "specs_beam_step_host": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32,
                                        _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -243,6 +248,34 @@ class Context:
             _ptr(tok_logprob), _ptr(blk_logprob_f64), _ptr(gen_blk_logprob_f64), _ptr(weights), _ptr(chosen),
             _ptr(accept), _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
             _stream()), "specs_beam_step")
+
+    def beam_step_dual_workspace_bytes(self, rows: int, d_target: int, d_gen: int, V: int) -> int:
+        return int(self._lib.specs_beam_step_dual_workspace_bytes(self._h, rows, d_target, d_gen, V))
+
+    def specs_beam_step_dual(self, hidden_target, w_target, hidden_gen, w_gen, token_ids, block_offsets, cand_offsets,
+                             reward, uniforms, beta, tau, tok_logprob, gen_tok_logprob, blk_logprob_f64,
+                             gen_blk_logprob_f64, weights, chosen, accept, workspace, chosen_ids=None,
+                             chosen_len=None):
+        """The step with both LM heads computed on the device (generator pass, target pass, finish kernel)."""
+        rows, d_t = hidden_target.shape
+        d_g = hidden_gen.shape[1]
+        V = w_target.shape[0]
+        B = block_offsets.shape[0] - 1
+        P = cand_offsets.shape[0] - 1
+        stride = 0 if chosen_ids is None else chosen_ids.shape[1]
+        _check(self._lib.specs_beam_step_dual(
+            self._h, _ptr(hidden_target), _ptr(w_target), d_t, _ptr(hidden_gen), _ptr(w_gen), d_g, _ptr(token_ids),
+            _ptr(block_offsets), _ptr(cand_offsets), _ptr(reward), _ptr(uniforms), rows, V, B, P, float(beta),
+            float(tau), _ptr(tok_logprob), _ptr(gen_tok_logprob), _ptr(blk_logprob_f64), _ptr(gen_blk_logprob_f64),
+            _ptr(weights), _ptr(chosen), _ptr(accept), _ptr(chosen_ids), _ptr(chosen_len), stride, _ptr(workspace),
+            0 if workspace is None else workspace.numel() * workspace.element_size(), _stream()),
+            "specs_beam_step_dual")
+
+    def specs_gather_chosen(self, token_ids, block_offsets, cand_offsets, chosen, chosen_ids, chosen_len):
+        P = cand_offsets.shape[0] - 1
+        _check(self._lib.specs_gather_chosen(self._h, _ptr(token_ids), _ptr(block_offsets), _ptr(cand_offsets),
+                                             _ptr(chosen), P, _ptr(chosen_ids), _ptr(chosen_len),
+                                             chosen_ids.shape[1], _stream()), "specs_gather_chosen")
 
     def specs_beam_step_host(self, h_hidden, w_vocab, h_token_ids, h_block_offsets, h_cand_offsets,
                              h_gen_tok_logprob, h_reward, h_uniforms, beta, tau,

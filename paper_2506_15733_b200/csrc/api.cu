@@ -402,9 +402,82 @@ int specs_beam_step(specs_ctx* ctx, const void* hidden, const void* W_vocab, con
         st = launch_score_tcgen05(ctx, plan, hidden, W_vocab, token_ids, static_cast<float*>(workspace), stream);
         if (st != SPECS_OK) return st;
     }
-    return launch_finish_step(ctx, plan, static_cast<const float*>(workspace), token_ids, block_offsets, cand_offsets,
-                              P, gen_tok_logprob, reward, uniforms, beta, tau, tok_logprob, blk_logprob_f64,
-                              gen_blk_logprob_f64, weights, chosen, accept, stream);
+    // the finish kernel only reads the generator's log-probabilities on this route
+    return launch_finish_step(ctx, plan, static_cast<const float*>(workspace), nullptr, nullptr, token_ids,
+                              block_offsets, cand_offsets, P, const_cast<float*>(gen_tok_logprob), reward, uniforms,
+                              beta, tau, tok_logprob, blk_logprob_f64, gen_blk_logprob_f64, weights, chosen, accept,
+                              nullptr, nullptr, 0, stream);
+}
+
+size_t specs_beam_step_dual_workspace_bytes(const specs_ctx* ctx, int64_t rows, int32_t d_target, int32_t d_gen,
+                                            int32_t V) {
+    const size_t t = specs_score_workspace_bytes(ctx, rows, d_target, V);
+    const size_t g = specs_score_workspace_bytes(ctx, rows, d_gen, V);
+    if (t == 0 || g == 0) return 0;
+    return ((t + 255) & ~(size_t)255) + g;
+}
+
+int specs_beam_step_dual(specs_ctx* ctx, const void* hidden_target, const void* W_target, int32_t d_target,
+                         const void* hidden_gen, const void* W_gen, int32_t d_gen, const int32_t* token_ids,
+                         const int64_t* block_offsets, const int32_t* cand_offsets, const float* reward,
+                         const float* uniforms, int64_t rows, int32_t V, int32_t B, int32_t P, float beta, float tau,
+                         float* tok_logprob, float* gen_tok_logprob, double* blk_logprob_f64,
+                         double* gen_blk_logprob_f64, float* weights, int32_t* chosen, uint8_t* accept,
+                         int32_t* chosen_ids, int32_t* chosen_len, int32_t chosen_stride, void* workspace,
+                         size_t workspace_bytes, void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    int st = check_score_shapes(rows, d_target, V, B);
+    if (st != SPECS_OK) return st;
+    if ((st = check_score_shapes(rows, d_gen, V, B)) != SPECS_OK) return st;
+    if (P < 0 || (chosen_ids && chosen_stride <= 0)) return SPECS_ERR_SHAPE;
+    if (P == 0) return SPECS_OK;
+    if (!W_target || !W_gen || !block_offsets || !cand_offsets || !chosen || (chosen_ids && !chosen_len))
+        return SPECS_ERR_NULL;
+    if (rows > 0 && (!hidden_target || !hidden_gen || !token_ids || !tok_logprob || !gen_tok_logprob || !workspace))
+        return SPECS_ERR_NULL;
+    if (B > 0 && (!reward || !uniforms || !blk_logprob_f64 || !gen_blk_logprob_f64)) return SPECS_ERR_NULL;
+    if (!aligned16(hidden_target) || !aligned16(W_target) || !aligned16(hidden_gen) || !aligned16(W_gen) ||
+        !aligned16(workspace))
+        return SPECS_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+    if (ctx->engine == SPECS_ENGINE_SIMT) return SPECS_ERR_SHAPE;
+
+    const int cta_group = ctx->engine == SPECS_ENGINE_TCGEN05_1CTA ? 1
+                        : ctx->engine == SPECS_ENGINE_TCGEN05_2CTA ? 2 : kCtaGroupAuto;
+    const ScorePlan plan_t = make_score_plan(rows, d_target, V, ctx->num_sms, ctx->pair_units, cta_group,
+                                             ctx->chunk_kblocks, ctx->accum_adaptive);
+    const ScorePlan plan_g = make_score_plan(rows, d_gen, V, ctx->num_sms, ctx->pair_units, cta_group,
+                                             ctx->chunk_kblocks, ctx->accum_adaptive);
+    const size_t off_g = (plan_workspace_bytes(plan_t) + 255) & ~(size_t)255;
+    float* ws_t = static_cast<float*>(workspace);
+    float* ws_g = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + off_g);
+    if (rows > 0) {
+        if (workspace_bytes < off_g + plan_workspace_bytes(plan_g)) return SPECS_ERR_WORKSPACE;
+        // the generator's (smaller) head first; both passes are done when the finish kernel starts
+        st = launch_score_tcgen05(ctx, plan_g, hidden_gen, W_gen, token_ids, ws_g, stream);
+        if (st != SPECS_OK) return st;
+        st = launch_score_tcgen05(ctx, plan_t, hidden_target, W_target, token_ids, ws_t, stream);
+        if (st != SPECS_OK) return st;
+    }
+    return launch_finish_step(ctx, plan_t, ws_t, &plan_g, rows > 0 ? ws_g : nullptr, token_ids, block_offsets,
+                              cand_offsets, P, gen_tok_logprob, reward, uniforms, beta, tau, tok_logprob,
+                              blk_logprob_f64, gen_blk_logprob_f64, weights, chosen, accept, chosen_ids, chosen_len,
+                              chosen_stride, stream);
+}
+
+int specs_gather_chosen(specs_ctx* ctx, const int32_t* token_ids, const int64_t* block_offsets,
+                        const int32_t* cand_offsets, const int32_t* chosen, int32_t P, int32_t* chosen_ids,
+                        int32_t* chosen_len, int32_t chosen_stride, void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    if (P < 0 || chosen_stride <= 0) return SPECS_ERR_SHAPE;
+    if (P == 0) return SPECS_OK;
+    if (!block_offsets || !cand_offsets || !chosen || !chosen_ids || !chosen_len) return SPECS_ERR_NULL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+    return launch_gather_chosen(token_ids, block_offsets, cand_offsets, chosen, P, chosen_ids, chosen_len,
+                                chosen_stride, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int specs_device_status(specs_ctx* ctx, uint32_t* h_bits, void* cuda_stream) {

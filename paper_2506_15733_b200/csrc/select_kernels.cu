@@ -254,13 +254,44 @@ __global__ void select_kernel(const double* __restrict__ lp_t, const double* __r
 // travel through the output arrays blk_lp / gen_lp (double).  One launch instead of four.
 constexpr int kFinishThreads = 1024;
 
+// Ids of the selected block of problem p into row p of chosen_ids [P, stride] (-1 beyond the block's
+// length, the whole row -1 when nothing was selected) and its length into chosen_len[p]: what Step II
+// of Algorithm 1 appends to the trace.  Executed by all threads of a CTA (or a warp with nthreads = 32).
+__device__ __forceinline__ void gather_chosen_block(const int32_t* __restrict__ token_ids,
+                                                    const int64_t* __restrict__ block_offsets, int a, int pick, int p,
+                                                    int32_t* __restrict__ chosen_ids, int32_t* __restrict__ chosen_len,
+                                                    int32_t stride, int tid, int nthreads) {
+    int64_t t0 = 0, len = 0;
+    if (pick >= 0) {
+        t0 = block_offsets[a + pick];
+        len = block_offsets[a + pick + 1] - t0;
+        if (len > stride) len = stride;                      // the host has checked that no block is longer
+    }
+    for (int k = tid; k < stride; k += nthreads)
+        chosen_ids[(size_t)p * stride + k] = k < len ? token_ids[t0 + k] : -1;
+    if (tid == 0) chosen_len[p] = (int32_t)len;
+}
+
+__global__ void gather_chosen_kernel(const int32_t* __restrict__ token_ids, const int64_t* __restrict__ block_offsets,
+                                     const int32_t* __restrict__ cand_offsets, const int32_t* __restrict__ chosen,
+                                     int32_t* __restrict__ chosen_ids, int32_t* __restrict__ chosen_len,
+                                     int32_t stride) {
+    const int p = blockIdx.x;
+    gather_chosen_block(token_ids, block_offsets, cand_offsets[p], chosen[p], p, chosen_ids, chosen_len, stride,
+                        threadIdx.x, blockDim.x);
+}
+
+// With workspace_g the generator's per-token log-probabilities are not an input: they are merged from
+// a second scoring pass (the generator's own LM head on the same drafted ids) and written to gen_tok.
 __global__ void __launch_bounds__(kFinishThreads)
-finish_step_kernel(const ScorePlan plan, const float* __restrict__ workspace, const int32_t* __restrict__ token_ids,
+finish_step_kernel(const ScorePlan plan, const float* __restrict__ workspace, const ScorePlan plan_g,
+                   const float* __restrict__ workspace_g, const int32_t* __restrict__ token_ids,
                    const int64_t* __restrict__ block_offsets, const int32_t* __restrict__ cand_offsets,
-                   const float* __restrict__ gen_tok_logprob, const float* __restrict__ reward,
-                   const float* __restrict__ uniforms, float beta, float tau, float* __restrict__ tok_logprob,
-                   double* blk_lp, double* gen_lp, float* __restrict__ weights, int32_t* __restrict__ chosen,
-                   uint8_t* __restrict__ accept, uint32_t* __restrict__ status) {
+                   float* gen_tok, const float* __restrict__ reward, const float* __restrict__ uniforms, float beta,
+                   float tau, float* __restrict__ tok_logprob, double* blk_lp, double* gen_lp,
+                   float* __restrict__ weights, int32_t* chosen, uint8_t* __restrict__ accept,
+                   int32_t* __restrict__ chosen_ids, int32_t* __restrict__ chosen_len, int32_t chosen_stride,
+                   uint32_t* __restrict__ status) {
     // Launched with programmatic stream serialisation: wait here for the scoring kernel's results.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int p = blockIdx.x;
@@ -268,15 +299,18 @@ finish_step_kernel(const ScorePlan plan, const float* __restrict__ workspace, co
     const int a = cand_offsets[p], b = cand_offsets[p + 1];
     if (b > a) {
         const int64_t row_a = block_offsets[a], row_b = block_offsets[b];   // the problem's rows are contiguous
-        for (int64_t row = row_a + threadIdx.x; row < row_b; row += kFinishThreads)
-            tok_logprob[row] = merged_logprob(plan, workspace, row, token_ids[row], status);
+        for (int64_t row = row_a + threadIdx.x; row < row_b; row += kFinishThreads) {
+            const int32_t id = token_ids[row];
+            tok_logprob[row] = merged_logprob(plan, workspace, row, id, status);
+            if (workspace_g) gen_tok[row] = merged_logprob(plan_g, workspace_g, row, id, status);
+        }
         __syncthreads();
         for (int i = a + warp; i < b; i += kFinishThreads / 32) {
             const int64_t t0 = block_offsets[i], t1 = block_offsets[i + 1];
             double lp = 0.0, lq = 0.0;
             for (int64_t t = t0 + lane; t < t1; t += 32) {
                 lp += (double)tok_logprob[t];
-                if (gen_tok_logprob) lq += (double)gen_tok_logprob[t];
+                if (gen_tok) lq += (double)gen_tok[t];
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
@@ -285,14 +319,19 @@ finish_step_kernel(const ScorePlan plan, const float* __restrict__ workspace, co
             }
             if (lane == 0) {
                 blk_lp[i] = lp;
-                if (gen_tok_logprob) gen_lp[i] = lq;
+                if (gen_tok) gen_lp[i] = lq;
             }
         }
         __syncthreads();
     }
     if (warp == 0)
-        subsample_problem<double>(blk_lp, gen_tok_logprob ? gen_lp : nullptr, reward, a, b, p, lane, beta, uniforms,
+        subsample_problem<double>(blk_lp, gen_tok ? gen_lp : nullptr, reward, a, b, p, lane, beta, uniforms,
                                   chosen, weights, tau, accept);
+    if (chosen_ids) {
+        __syncthreads();                                      // chosen[p] was written by warp 0 of this CTA
+        gather_chosen_block(token_ids, block_offsets, a, chosen[p], p, chosen_ids, chosen_len, chosen_stride,
+                            threadIdx.x, kFinishThreads);
+    }
 }
 
 __global__ void accept_kernel(const float* __restrict__ reward, const int32_t* __restrict__ cand_offsets, int32_t P,
@@ -323,11 +362,12 @@ int launch_merge(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, 
     return cuda_status(cudaGetLastError());
 }
 
-int launch_finish_step(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, const int32_t* token_ids,
-                       const int64_t* block_offsets, const int32_t* cand_offsets, int32_t P,
-                       const float* gen_tok_logprob, const float* reward, const float* uniforms, float beta, float tau,
-                       float* tok_logprob, double* blk_lp, double* gen_lp, float* weights, int32_t* chosen,
-                       uint8_t* accept, cudaStream_t stream) {
+int launch_finish_step(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, const ScorePlan* plan_g,
+                       const float* workspace_g, const int32_t* token_ids, const int64_t* block_offsets,
+                       const int32_t* cand_offsets, int32_t P, float* gen_tok, const float* reward,
+                       const float* uniforms, float beta, float tau, float* tok_logprob, double* blk_lp, double* gen_lp,
+                       float* weights, int32_t* chosen, uint8_t* accept, int32_t* chosen_ids, int32_t* chosen_len,
+                       int32_t chosen_stride, cudaStream_t stream) {
     if (P == 0) return SPECS_OK;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)P, 1, 1);
@@ -339,9 +379,20 @@ int launch_finish_step(specs_ctx* ctx, const ScorePlan& plan, const float* works
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cuda_status(cudaLaunchKernelEx(&cfg, finish_step_kernel, plan, workspace, token_ids, block_offsets,
-                                          cand_offsets, gen_tok_logprob, reward, uniforms, beta, tau, tok_logprob,
-                                          blk_lp, gen_lp, weights, chosen, accept, ctx->d_status));
+    const ScorePlan second = plan_g ? *plan_g : plan;
+    return cuda_status(cudaLaunchKernelEx(&cfg, finish_step_kernel, plan, workspace, second, workspace_g, token_ids,
+                                          block_offsets, cand_offsets, gen_tok, reward, uniforms, beta, tau,
+                                          tok_logprob, blk_lp, gen_lp, weights, chosen, accept, chosen_ids, chosen_len,
+                                          chosen_stride, ctx->d_status));
+}
+
+int launch_gather_chosen(const int32_t* token_ids, const int64_t* block_offsets, const int32_t* cand_offsets,
+                         const int32_t* chosen, int32_t P, int32_t* chosen_ids, int32_t* chosen_len, int32_t stride,
+                         cudaStream_t stream) {
+    if (P == 0) return SPECS_OK;
+    gather_chosen_kernel<<<(unsigned)P, 128, 0, stream>>>(token_ids, block_offsets, cand_offsets, chosen, chosen_ids,
+                                                          chosen_len, stride);
+    return cuda_status(cudaGetLastError());
 }
 
 int launch_block_sums(const float* per_token, const int64_t* block_offsets, int32_t B, float* out, double* out_f64,

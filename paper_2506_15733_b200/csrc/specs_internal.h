@@ -126,11 +126,15 @@ int launch_score_simt(specs_ctx* ctx, const void* hidden, const void* w_vocab, c
                       int64_t rows, int32_t d, int32_t V, float* tok_logprob, cudaStream_t stream);
 int launch_merge(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, const int32_t* token_ids,
                  float* tok_logprob, cudaStream_t stream);
-int launch_finish_step(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, const int32_t* token_ids,
-                       const int64_t* block_offsets, const int32_t* cand_offsets, int32_t P,
-                       const float* gen_tok_logprob, const float* reward, const float* uniforms, float beta, float tau,
-                       float* tok_logprob, double* blk_lp, double* gen_lp, float* weights, int32_t* chosen,
-                       uint8_t* accept, cudaStream_t stream);
+int launch_finish_step(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, const ScorePlan* plan_g,
+                       const float* workspace_g, const int32_t* token_ids, const int64_t* block_offsets,
+                       const int32_t* cand_offsets, int32_t P, float* gen_tok, const float* reward,
+                       const float* uniforms, float beta, float tau, float* tok_logprob, double* blk_lp, double* gen_lp,
+                       float* weights, int32_t* chosen, uint8_t* accept, int32_t* chosen_ids, int32_t* chosen_len,
+                       int32_t chosen_stride, cudaStream_t stream);
+int launch_gather_chosen(const int32_t* token_ids, const int64_t* block_offsets, const int32_t* cand_offsets,
+                         const int32_t* chosen, int32_t P, int32_t* chosen_ids, int32_t* chosen_len, int32_t stride,
+                         cudaStream_t stream);
 int launch_block_sums(const float* per_token, const int64_t* block_offsets, int32_t B,
                       float* out, double* out_f64, cudaStream_t stream);
 int launch_subsample(const void* lp_target, const void* lp_gen, bool lp_is_f64, const float* reward,

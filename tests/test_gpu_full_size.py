@@ -164,6 +164,37 @@ def test_dual_scoring_draft_then_target(ctx, token_dist):
     assert check_selection_logic(x, g, 1.0, 0.7, blk["dual_draft"].cpu().numpy()) >= 6
 
 
+def test_dual_head_step_at_full_size(ctx):
+    # both heads in one call (generator pass, target pass, finish kernel) on the 65536 drafted tokens
+    from oracle import specs_variants as OV
+    xg = I.make_step_inputs(I.CONFIGS["dual_draft"])
+    xt = I.make_step_inputs(I.CONFIGS["dual_target"])
+    assert np.array_equal(xg.token_ids, xt.token_ids) and np.array_equal(xg.block_offsets, xt.block_offsets)
+    dev = "cuda:0"
+    s = DeviceStep(ctx, xt)
+    h_g, w_g = binding.bf16_bits_to_device(xg.hidden, dev), binding.bf16_bits_to_device(xg.w_vocab, dev)
+    gen_tok = torch.full((xt.rows,), float("nan"), dtype=torch.float32, device=dev)
+    ids_out = torch.full((8, 256), -9, dtype=torch.int32, device=dev)
+    len_out = torch.full((8,), -9, dtype=torch.int32, device=dev)
+    ws = torch.empty(ctx.beam_step_dual_workspace_bytes(xt.rows, 3584, 1536, 151936), dtype=torch.uint8, device=dev)
+    ctx.specs_beam_step_dual(s.hidden, s.w_vocab, h_g, w_g, s.token_ids, s.block_offsets, s.cand_offsets, s.reward,
+                             s.uniforms, 1.0, 0.7, s.tok_lp, gen_tok, s.blk_lp64, s.gen_blk64, s.weights, s.chosen,
+                             s.accept, ws, ids_out, len_out)
+    torch.cuda.synchronize()
+    got = s.results()
+    g_tok = gen_tok.cpu().numpy()
+    rng = np.random.Generator(np.random.Philox(key=[7005, 1]))
+    rows_idx = np.unique(np.concatenate([rows_of_blocks(xt, [5]), rng.choice(xt.rows, 96, replace=False)]))
+    check_sampled_rows(xt, got["tok_logprob"], rows_idx, O.bf16_bits_to_f64(xt.w_vocab))
+    check_sampled_rows(xg, g_tok, rows_idx, O.bf16_bits_to_f64(xg.w_vocab))
+    # block sums of both heads are the plain sums of the GPU's own token log-probs; selection logic on all problems
+    assert np.allclose(got["blk_logprob_f64"], O.block_sums(got["tok_logprob"], xt.block_offsets), rtol=1e-12)
+    assert np.allclose(got["blk_logprob_gen"], O.block_sums(g_tok, xt.block_offsets), rtol=1e-12)
+    assert check_selection_logic(xt, got, 1.0, 0.7, got["blk_logprob_gen"]) >= 6
+    want_ids, want_len = OV.gather_chosen(xt.token_ids, xt.block_offsets, xt.cand_offsets, got["chosen"], 256)
+    assert np.array_equal(ids_out.cpu().numpy(), want_ids) and np.array_equal(len_out.cpu().numpy(), want_len)
+
+
 def test_stress_heavy_tailed_logits(ctx):
     cfg = I.CONFIGS["stress"]
     x = I.make_step_inputs(cfg)

@@ -547,3 +547,57 @@ def test_specs_loop_with_stub_generators(ctx):
     st = got_ctl.stats()
     assert st["steps"].sum() >= P and (st["target_steps"] >= 1).all()   # every problem began with the target
     assert ctx.device_status() == 0
+
+
+# ------------------------------------------------------------------------------- both LM heads, and the append
+
+def test_dual_head_step_and_gather_match_the_oracle(ctx):
+    # the same drafted tokens scored with a small generator-shaped head and a larger target-shaped head
+    P, n, V_ = 5, 4, 2500
+    cfg_t = small_config("dual_t", (3, 70), P, n, 256, V_, seed=5600)
+    cfg_g = small_config("dual_g", (3, 70), P, n, 128, V_, seed=5600, w_sigma=0.07, weights_salt=1)
+    xt, xg = I.make_step_inputs(cfg_t), I.make_step_inputs(cfg_g)
+    assert np.array_equal(xt.block_offsets, xg.block_offsets) and np.array_equal(xt.token_ids, xg.token_ids)
+    xt.cand_offsets = np.array([0, 4, 8, 8, 12, 20], dtype=np.int32)                      # one empty problem
+    dev = "cuda:0"
+    s = DeviceStep(ctx, xt)
+    h_g, w_g = binding.bf16_bits_to_device(xg.hidden, dev), binding.bf16_bits_to_device(xg.w_vocab, dev)
+    gen_tok = torch.full((xt.rows,), float("nan"), dtype=torch.float32, device=dev)
+    stride = 72
+    ids_out = torch.full((P, stride), -9, dtype=torch.int32, device=dev)
+    len_out = torch.full((P,), -9, dtype=torch.int32, device=dev)
+    ws = torch.empty(ctx.beam_step_dual_workspace_bytes(xt.rows, 256, 128, V_), dtype=torch.uint8, device=dev)
+    ctx.specs_beam_step_dual(s.hidden, s.w_vocab, h_g, w_g, s.token_ids, s.block_offsets, s.cand_offsets, s.reward,
+                             s.uniforms, 1.0, 0.6, s.tok_lp, gen_tok, s.blk_lp64, s.gen_blk64, s.weights, s.chosen,
+                             s.accept, ws, ids_out, len_out)
+    torch.cuda.synchronize()
+    got = s.results()
+    got["blk_logprob"] = got["blk_logprob_f64"].astype(np.float32)
+    want = OV.beam_step_dual(xt.hidden, xt.w_vocab, xg.hidden, xg.w_vocab, xt.token_ids, xt.block_offsets,
+                             xt.cand_offsets, xt.reward, 1.0, xt.uniforms, 0.6)
+    assert_step_matches(got, want, xt.cand_offsets, xt.block_offsets)
+    g_tok = gen_tok.cpu().numpy()
+    assert np.abs(g_tok - want["gen_tok_logprob"]).max() <= TOK_ATOL
+    assert np.abs((got["tok_logprob"] - g_tok) - want["tok_logratio"]).max() <= 2 * TOK_ATOL   # per-token log-ratio
+    rel = np.abs(got["blk_logprob_gen"] - want["blk_logprob_gen"]) / np.abs(want["blk_logprob_gen"])
+    assert rel.max() <= BLK_RTOL
+    # the append: ids and length of the block the GPU selected, bit-exact against the definition
+    want_ids, want_len = OV.gather_chosen(xt.token_ids, xt.block_offsets, xt.cand_offsets, got["chosen"], stride)
+    assert np.array_equal(ids_out.cpu().numpy(), want_ids) and np.array_equal(len_out.cpu().numpy(), want_len)
+    assert got["chosen"][2] == -1 and want_len[2] == 0
+    # the stand-alone gather gives the same
+    ids2 = torch.full((P, stride), -9, dtype=torch.int32, device=dev)
+    len2 = torch.full((P,), -9, dtype=torch.int32, device=dev)
+    ctx.specs_gather_chosen(s.token_ids, s.block_offsets, s.cand_offsets, s.chosen, ids2, len2)
+    torch.cuda.synchronize()
+    assert torch.equal(ids2, ids_out) and torch.equal(len2, len_out)
+    # and the two-head step equals the one-head step fed with the generator's log-probs it computed
+    s2 = DeviceStep(ctx, xt)
+    ctx.specs_beam_step(s2.hidden, s2.w_vocab, s2.token_ids, s2.block_offsets, s2.cand_offsets, gen_tok, s2.reward,
+                        s2.uniforms, 1.0, 0.6, s2.tok_lp, s2.blk_lp64, s2.gen_blk64, s2.weights, s2.chosen, s2.accept,
+                        s2.workspace)
+    torch.cuda.synchronize()
+    one = s2.results()
+    for key in ("tok_logprob", "blk_logprob_f64", "blk_logprob_gen", "weights", "chosen", "accept"):
+        assert np.array_equal(one[key], got[key]), key
+    assert ctx.device_status() == 0
