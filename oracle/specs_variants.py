@@ -189,3 +189,29 @@ def gather_chosen(token_ids, block_offsets, cand_offsets, chosen, stride):
             out[p, k - a] = token_ids[k]
         lens[p] = b - a
     return out, lens
+
+
+# --------------------------------------------------------------------------- PRM head
+
+def prm_rewards(prm_hidden_bits, block_offsets, w_head_bits, bias):
+    """r(Y_i | tr) of every drafted block from the process reward model's final hidden states: the value
+    head (one weight vector and a bias) applied to the hidden state of the block's LAST token, squashed
+    to (0, 1) by the logistic function.  The paper takes r as given (Section 2: "PRM r") and uses a PRM
+    whose scores are thresholded between 0.5 and 0.9, i.e. lie in [0, 1] (Section 4.1, Table 6); which
+    position is read and the logistic link are this build's reading.  An empty block has no last token:
+    its reward is NaN.  Inputs are bf16 bit patterns; everything is evaluated in float64."""
+    from oracle import specs_oracle as O
+    H = O.bf16_bits_to_f64(prm_hidden_bits)
+    w = O.bf16_bits_to_f64(w_head_bits)
+    b = float(np.float32(bias))
+    B = len(block_offsets) - 1
+    out = np.full(B, np.nan)
+    for i in range(B):
+        a, e = int(block_offsets[i]), int(block_offsets[i + 1])
+        if e <= a:
+            continue
+        z = b
+        for k in range(H.shape[1]):
+            z += H[e - 1, k] * w[k]
+        out[i] = 1.0 / (1.0 + np.exp(-z))
+    return out

@@ -213,3 +213,33 @@ def test_gather_chosen_worked_example():
     assert out[0].tolist() == [-1] * 4 and lens.tolist() == [0, 0, 4] and out[2].tolist() == [103, 104, 105, 106]
     with pytest.raises(ValueError):
         V.gather_chosen(ids, boff, cand, np.array([0, -1, 0]), 3)
+
+
+# ------------------------------------------------------------------------------- PRM head
+
+def test_prm_head_closed_forms():
+    from scipy.special import expit
+
+    def bits(a):
+        return (np.asarray(a, np.float32).view(np.uint32) >> 16).astype(np.uint16)
+    rng = np.random.Generator(np.random.Philox(key=[6900, 1]))
+    d, rows = 24, 9
+    H = rng.integers(-8, 9, (rows, d)) / 8.0                     # exact in bf16
+    w = rng.integers(-8, 9, d) / 16.0
+    boff = np.array([0, 2, 2, 5, 9])
+    r = V.prm_rewards(bits(H), boff, bits(w), 0.25)
+    last = [1, None, 4, 8]                                        # the block's LAST token is read
+    for i, t in enumerate(last):
+        if t is None:
+            assert np.isnan(r[i])                                 # an empty block has no last token
+        else:
+            assert abs(r[i] - expit(float(H[t] @ w) + 0.25)) < 1e-15
+    assert np.all((r[[0, 2, 3]] > 0) & (r[[0, 2, 3]] < 1))
+    # zero hidden state: the logistic of the bias alone; zero weight too: exactly one half
+    assert V.prm_rewards(bits(np.zeros((1, d))), np.array([0, 1]), bits(w), 0.25)[0] == expit(0.25)
+    assert V.prm_rewards(bits(H[:1]), np.array([0, 1]), bits(np.zeros(d)), 0.0)[0] == 0.5
+    # sigma(-z) = 1 - sigma(z): negating the head mirrors the reward
+    r_neg = V.prm_rewards(bits(H), boff, bits(-w), -0.25)
+    assert np.allclose(r_neg[[0, 2, 3]], 1.0 - r[[0, 2, 3]], rtol=0, atol=1e-15)
+    # monotone in the bias
+    assert np.all(V.prm_rewards(bits(H), boff, bits(w), 1.0)[[0, 2, 3]] > r[[0, 2, 3]])
