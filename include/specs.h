@@ -218,6 +218,20 @@ int specs_select(specs_ctx* ctx, const double* blk_lp_target, const double* blk_
                  int switch_rule, float tau, int32_t* chosen, float* weights, uint8_t* flag,
                  void* cuda_stream);
 
+/* Rewards r(Y_i | tr) of the drafted blocks from the process reward model's final
+ * hidden states (Section 2 takes the PRM r as given; Appendix E.3 evaluates it
+ * concurrently with the target's log-likelihoods, which a caller gets by issuing
+ * this call on a second stream):
+ *   reward[i] = 1 / (1 + exp(-(w_head . h_last(i) + bias)))
+ * where h_last(i) is row block_offsets[i+1] - 1 of prm_hidden, the hidden state at the
+ * block's last token.  The logistic link and the position read are this library's
+ * reading of a value-head PRM whose scores lie in [0, 1]; an empty block has no last
+ * token and gets NaN.
+ *   prm_hidden bf16 [rows, d] row-major, w_head bf16 [d], both 16-byte aligned,
+ *   d % 8 == 0; block_offsets int64 [B+1] on the device; reward float [B] out. */
+int specs_prm_rewards(specs_ctx* ctx, const void* prm_hidden, const int64_t* block_offsets, int32_t B,
+                      int32_t d, const void* w_head, float bias, float* reward, void* cuda_stream);
+
 /* The dynamic-switching test alone (Algorithm 1, Step III; Section 2.3):
  * accept[p] = 1 iff the largest reward among ALL candidates of problem p is
  * strictly above tau, i.e. the draft model may generate the next step.  The call

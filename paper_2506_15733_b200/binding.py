@@ -50,6 +50,7 @@ SIGNATURES = {
     "specs_subsample": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _f32, _vp, _vp, _vp, _f32, _vp, _vp]),
     "specs_subsample_f64": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _f32, _vp, _vp, _vp, _f32, _vp, _vp]),
     "specs_accept": (C.c_int, [_vp, _vp, _vp, _i32, _f32, _vp, _vp]),
+    "specs_prm_rewards": (C.c_int, [_vp, _vp, _vp, _i32, _i32, _vp, _f32, _vp, _vp]),
     "specs_select": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _f32, _vp, C.c_int, C.c_int, C.c_int, _f32,
                                _vp, _vp, _vp, _vp]),
     "specs_controller_create": (C.c_int, [C.POINTER(_vp), _i32, _vp]),
@@ -224,6 +225,12 @@ class Context:
         P = cand_offsets.shape[0] - 1
         _check(self._lib.specs_accept(self._h, _ptr(reward), _ptr(cand_offsets), P, float(tau), _ptr(accept),
                                       _stream()), "specs_accept")
+
+    def specs_prm_rewards(self, prm_hidden, block_offsets, w_head, bias, reward):
+        """Value head of the PRM on each block's last hidden state, logistic link; reward float32 [B] out."""
+        B = block_offsets.shape[0] - 1
+        _check(self._lib.specs_prm_rewards(self._h, _ptr(prm_hidden), _ptr(block_offsets), B, prm_hidden.shape[1],
+                                           _ptr(w_head), float(bias), _ptr(reward), _stream()), "specs_prm_rewards")
 
     def specs_select(self, blk_lp_target, blk_lp_gen, reward, mask, cand_offsets, beta, uniforms, select_rule,
                      score_flags, switch_rule, tau, chosen, weights=None, flag=None):

@@ -361,6 +361,19 @@ int specs_select(specs_ctx* ctx, const double* blk_lp_target, const double* blk_
                          score_flags, switch_rule, tau, chosen, weights, flag, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int specs_prm_rewards(specs_ctx* ctx, const void* prm_hidden, const int64_t* block_offsets, int32_t B, int32_t d,
+                      const void* w_head, float bias, float* reward, void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    if (B < 0 || d <= 0 || (d % 8) != 0) return SPECS_ERR_SHAPE;
+    if (B == 0) return SPECS_OK;
+    if (!prm_hidden || !block_offsets || !w_head || !reward) return SPECS_ERR_NULL;
+    if (!aligned16(prm_hidden) || !aligned16(w_head)) return SPECS_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+    return launch_prm_head(prm_hidden, block_offsets, B, d, w_head, bias, reward,
+                           static_cast<cudaStream_t>(cuda_stream));
+}
+
 int specs_accept(specs_ctx* ctx, const float* reward, const int32_t* cand_offsets, int32_t P, float tau,
                  uint8_t* accept, void* cuda_stream) {
     if (!ctx) return SPECS_ERR_NULL;

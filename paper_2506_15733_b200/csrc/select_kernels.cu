@@ -8,6 +8,8 @@
 //                         switch test of Algorithm 1, Step III;
 //   accept_kernel         the switch test alone;
 //   finish_step_kernel    all of the above for one problem per CTA, for the fused beam step.
+#include <cuda_bf16.h>
+
 #include "specs_internal.h"
 
 namespace specs {
@@ -334,6 +336,42 @@ finish_step_kernel(const ScorePlan plan, const float* __restrict__ workspace, co
     }
 }
 
+// ------------------------------------------------------------------------------------ PRM head
+// Reward of every drafted block from the process reward model's final hidden states: the value head
+// (one weight vector, one bias) on the hidden state of the block's last token, through the logistic
+// function.  One warp per block; 16-byte loads of eight bf16 at a time, fp32 products summed in fp32
+// per lane and in double across the lanes.  HBM-bound on B rows of d bf16 (plus the head, from L2).
+__global__ void prm_head_kernel(const __nv_bfloat16* __restrict__ prm_hidden, const int64_t* __restrict__ block_offsets,
+                                int32_t B, int32_t d, const __nv_bfloat16* __restrict__ w_head, float bias,
+                                float* __restrict__ reward) {
+    const int i = (int)(((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+    const int lane = threadIdx.x & 31;
+    if (i >= B) return;
+    const int64_t a = block_offsets[i], e = block_offsets[i + 1];
+    if (e <= a) {                                            // no last token
+        if (lane == 0) reward[i] = __int_as_float(0x7fc00000);
+        return;
+    }
+    const uint4* h = reinterpret_cast<const uint4*>(prm_hidden + (size_t)(e - 1) * d);
+    const uint4* w = reinterpret_cast<const uint4*>(w_head);
+    float acc = 0.0f;
+    for (int v = lane; v < d / 8; v += 32) {
+        const uint4 hv = __ldg(h + v), wv = __ldg(w + v);
+        const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hv);
+        const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float2 x = __bfloat1622float2(hp[j]), y = __bfloat1622float2(wp[j]);
+            acc = fmaf(x.x, y.x, acc);
+            acc = fmaf(x.y, y.y, acc);
+        }
+    }
+    double z = (double)acc;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(kFull, z, o);
+    if (lane == 0) reward[i] = (float)(1.0 / (1.0 + exp(-(z + (double)bias))));
+}
+
 __global__ void accept_kernel(const float* __restrict__ reward, const int32_t* __restrict__ cand_offsets, int32_t P,
                               float tau, uint8_t* __restrict__ accept) {
     const int p = (int)(((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
@@ -429,6 +467,16 @@ int launch_select(const double* lp_target, const double* lp_gen, const float* re
     select_kernel<<<warps_grid(P, threads), threads, 0, stream>>>(lp_target, lp_gen, reward, mask, cand_offsets, P,
                                                                    beta, uniforms, select_rule, score_flags,
                                                                    switch_rule, tau, chosen, weights, flag);
+    return cuda_status(cudaGetLastError());
+}
+
+int launch_prm_head(const void* prm_hidden, const int64_t* block_offsets, int32_t B, int32_t d, const void* w_head,
+                    float bias, float* reward, cudaStream_t stream) {
+    if (B == 0) return SPECS_OK;
+    const int threads = 128;
+    prm_head_kernel<<<warps_grid(B, threads), threads, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(prm_hidden), block_offsets, B, d, static_cast<const __nv_bfloat16*>(w_head),
+        bias, reward);
     return cuda_status(cudaGetLastError());
 }
 

@@ -144,6 +144,8 @@ int launch_select(const double* lp_target, const double* lp_gen, const float* re
                   const int32_t* cand_offsets, int32_t P, float beta, const float* uniforms, int select_rule,
                   int score_flags, int switch_rule, float tau, int32_t* chosen, float* weights, uint8_t* flag,
                   cudaStream_t stream);
+int launch_prm_head(const void* prm_hidden, const int64_t* block_offsets, int32_t B, int32_t d, const void* w_head,
+                    float bias, float* reward, cudaStream_t stream);
 int launch_accept(const float* reward, const int32_t* cand_offsets, int32_t P, float tau,
                   uint8_t* accept, cudaStream_t stream);
 

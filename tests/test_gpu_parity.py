@@ -601,3 +601,38 @@ def test_dual_head_step_and_gather_match_the_oracle(ctx):
     for key in ("tok_logprob", "blk_logprob_f64", "blk_logprob_gen", "weights", "chosen", "accept"):
         assert np.array_equal(one[key], got[key]), key
     assert ctx.device_status() == 0
+
+
+# ------------------------------------------------------------------------------- PRM head
+
+def test_prm_head_matches_the_oracle_and_overlaps_with_scoring(ctx):
+    cfg = small_config("prm", (0, 60), 6, 8, 3584, 520, seed=5700)   # blocks of 0..60 tokens, some empty
+    x = I.make_step_inputs(cfg)
+    assert (np.diff(x.block_offsets) == 0).any()
+    rng = np.random.Generator(np.random.Philox(key=[5701, 1]))
+    w_head = I.f32_to_bf16_bits((rng.normal(0, 0.03, 3584)).astype(np.float32))
+    dev = "cuda:0"
+    s = DeviceStep(ctx, x)
+    w_dev = binding.bf16_bits_to_device(w_head.reshape(1, -1), dev).reshape(-1)
+    reward = torch.full((x.blocks,), -3.0, dtype=torch.float32, device=dev)
+    # the paper evaluates the PRM concurrently with the target's log-likelihoods: second stream
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        ctx.specs_prm_rewards(s.hidden, s.block_offsets, w_dev, -0.4, reward)
+    s.score()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    want = OV.prm_rewards(x.hidden, x.block_offsets, w_head, -0.4)
+    got = reward.cpu().numpy()
+    empty = np.diff(x.block_offsets) == 0
+    assert np.isnan(got[empty]).all() and np.isnan(want[empty]).all()
+    assert np.abs(got[~empty] - want[~empty]).max() < 2e-6           # fp32 dot over 3584 terms, fp32 output
+    assert want[~empty].min() > 0.01 and want[~empty].max() < 0.99 and np.ptp(want[~empty]) > 0.3
+    # scoring on the main stream was not disturbed
+    assert np.abs(s.tok_lp.cpu().numpy() - O.token_logprobs(x.hidden, x.w_vocab, x.token_ids)).max() <= TOK_ATOL
+    # argument checks
+    with pytest.raises(binding.SpecsError) as e:
+        ctx.specs_prm_rewards(s.hidden[:, :12], s.block_offsets, w_dev, 0.0, reward)
+    assert e.value.status == 2
+    assert ctx.device_status() == 0
