@@ -215,3 +215,37 @@ def prm_rewards(prm_hidden_bits, block_offsets, w_head_bits, bias):
             z += H[e - 1, k] * w[k]
         out[i] = 1.0 / (1.0 + np.exp(-z))
     return out
+
+
+# --------------------------------------------------------------------------- vocabulary shards
+
+def shard_partials(hidden_bits, w_bits, token_ids, v0, v1):
+    """What one holder of vocabulary rows [v0, v1) can say about every drafted row: the largest logit of its
+    shard, the sum of exp(logit - that maximum) over the shard, and the drafted id's logit if the id lies in
+    the shard (-inf otherwise).  float64 [rows, 3]."""
+    from oracle import specs_oracle as O
+    H = O.bf16_bits_to_f64(hidden_bits)
+    W = O.bf16_bits_to_f64(w_bits[v0:v1])
+    out = np.empty((H.shape[0], 3))
+    for t in range(H.shape[0]):
+        z = W @ H[t]
+        m = np.max(z)
+        y = int(token_ids[t])
+        out[t] = (m, np.sum(np.exp(z - m)), z[y - v0] if v0 <= y < v1 else -np.inf)
+    return out
+
+
+def merge_partials(partials, token_ids, V):
+    """log pi_target(y_t) from the shards' partials: the log-sum-exp of a union is the log-sum-exp of the
+    parts' log-sum-exps; the drafted id's logit is held by exactly one shard.  partials float64 [g, rows, 3]."""
+    partials = np.asarray(partials, dtype=np.float64)
+    g, rows, _ = partials.shape
+    out = np.empty(rows)
+    for t in range(rows):
+        M = np.max(partials[:, t, 0])
+        total = 0.0
+        for j in range(g):
+            total += partials[j, t, 1] * np.exp(partials[j, t, 0] - M)
+        y = int(token_ids[t])
+        out[t] = np.max(partials[:, t, 2]) - (M + np.log(total)) if 0 <= y < V else np.nan
+    return out

@@ -243,3 +243,24 @@ def test_prm_head_closed_forms():
     assert np.allclose(r_neg[[0, 2, 3]], 1.0 - r[[0, 2, 3]], rtol=0, atol=1e-15)
     # monotone in the bias
     assert np.all(V.prm_rewards(bits(H), boff, bits(w), 1.0)[[0, 2, 3]] > r[[0, 2, 3]])
+
+
+# ------------------------------------------------------------------------------- vocabulary shards
+
+@pytest.mark.parametrize("cuts", [(0, 37), (0, 1, 37), (0, 5, 20, 21, 37), (0, 36, 37)])
+def test_sharded_log_softmax_equals_the_whole(cuts):
+    # the log-sum-exp over a partition of the vocabulary, against the unsharded definition
+    cfg = I.StepConfig("shards", 7100, 1, 3, (4, 4), 16, 37, 0.6, hidden_scale=2.0)
+    x = I.make_step_inputs(cfg)
+    ids = x.token_ids.copy()
+    ids[0], ids[1] = 0, 36                                        # first and last vocabulary entry
+    whole = O.token_logprobs(x.hidden, x.w_vocab, ids)
+    parts = np.stack([V.shard_partials(x.hidden, x.w_vocab, ids, a, b) for a, b in zip(cuts[:-1], cuts[1:])])
+    assert np.allclose(V.merge_partials(parts, ids, 37), whole, rtol=0, atol=1e-12)
+    assert np.all((parts[:, :, 2] > -np.inf).sum(axis=0) == 1)    # exactly one shard holds the drafted id
+    # the order of the shards does not matter
+    assert np.allclose(V.merge_partials(parts[::-1], ids, 37), whole, rtol=0, atol=1e-12)
+    # an id outside the vocabulary has no probability
+    bad = ids.copy(); bad[2] = 37
+    parts_bad = np.stack([V.shard_partials(x.hidden, x.w_vocab, bad, a, b) for a, b in zip(cuts[:-1], cuts[1:])])
+    assert np.isnan(V.merge_partials(parts_bad, bad, 37)[2])
