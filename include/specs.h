@@ -302,6 +302,28 @@ int specs_gather_chosen(specs_ctx* ctx, const int32_t* token_ids, const int64_t*
                         const int32_t* cand_offsets, const int32_t* chosen, int32_t P,
                         int32_t* chosen_ids, int32_t* chosen_len, int32_t chosen_stride, void* cuda_stream);
 
+/* Vocabulary-parallel scoring: each holder of a shard of W_vocab (rows id_offset ..
+ * id_offset + V_shard - 1 of the whole matrix) scores all drafted rows against its
+ * shard and produces, per row, what the log-softmax needs from it:
+ *   partials[row] = { max logit of the shard * log2(e),
+ *                     sum over the shard of 2^(logit*log2(e) - that maximum),
+ *                     the drafted id's logit if id_offset <= id < id_offset + V_shard,
+ *                       else -inf,
+ *                     0 }                                   (float [rows, 4], 16-byte aligned)
+ * token_ids are indices into the WHOLE vocabulary; an id outside the shard is not an
+ * error here.  The partials of all shards (e.g. all-gathered over NVLink into
+ * [shards, rows, 4]) are folded by specs_merge_partials into log pi_target of the
+ * drafted id (Section 2; the log-sum-exp over a partition is the log-sum-exp of the
+ * parts), NaN and SPECS_DEV_TOKEN_RANGE for an id outside [0, V).  This is the paper's
+ * scoring step cut the other way than by rows; the paper itself places each model on
+ * one GPU (Appendix E.2).  Workspace as for specs_score_blocks with V = V_shard. */
+int specs_score_partials(specs_ctx* ctx, const void* hidden, const void* W_shard,
+                         const int32_t* token_ids, int32_t id_offset, int64_t rows, int32_t d,
+                         int32_t V_shard, float* partials, void* workspace, size_t workspace_bytes,
+                         void* cuda_stream);
+int specs_merge_partials(specs_ctx* ctx, const float* partials, int32_t shards, int64_t rows,
+                         const int32_t* token_ids, int32_t V, float* tok_logprob, void* cuda_stream);
+
 /* Host-side controller of the SPECS loop (Algorithm 1): for P problems it keeps which
  * model drafts the next n candidate blocks, appends the selected block, applies the
  * dynamic switch (Step III; Section 2.3) and stops at the target length.  All

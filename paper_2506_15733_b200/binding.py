@@ -46,6 +46,8 @@ SIGNATURES = {
     "specs_score_workspace_bytes": (C.c_size_t, [_vp, _i64, _i32, _i32]),
     "specs_score_blocks": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp,
                                      C.c_size_t, _vp]),
+    "specs_score_partials": (C.c_int, [_vp, _vp, _vp, _vp, _i32, _i64, _i32, _i32, _vp, _vp, C.c_size_t, _vp]),
+    "specs_merge_partials": (C.c_int, [_vp, _vp, _i32, _i64, _vp, _i32, _vp, _vp]),
     "specs_block_sums": (C.c_int, [_vp, _vp, _vp, _i32, _vp, _vp, _vp]),
     "specs_subsample": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _f32, _vp, _vp, _vp, _f32, _vp, _vp]),
     "specs_subsample_f64": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _f32, _vp, _vp, _vp, _f32, _vp, _vp]),
@@ -225,6 +227,20 @@ class Context:
         P = cand_offsets.shape[0] - 1
         _check(self._lib.specs_accept(self._h, _ptr(reward), _ptr(cand_offsets), P, float(tau), _ptr(accept),
                                       _stream()), "specs_accept")
+
+    def specs_score_partials(self, hidden, w_shard, token_ids, id_offset, partials, workspace):
+        """Per-row (max, sum, logit) of one vocabulary shard; partials float32 [rows, 4] out."""
+        rows, d = hidden.shape
+        _check(self._lib.specs_score_partials(
+            self._h, _ptr(hidden), _ptr(w_shard), _ptr(token_ids), int(id_offset), rows, d, w_shard.shape[0],
+            _ptr(partials), _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
+            "specs_score_partials")
+
+    def specs_merge_partials(self, partials, token_ids, V, tok_logprob):
+        """Fold the shards' partials float32 [shards, rows, 4] into log pi_target of the drafted ids."""
+        shards, rows = partials.shape[0], partials.shape[1]
+        _check(self._lib.specs_merge_partials(self._h, _ptr(partials), shards, rows, _ptr(token_ids), int(V),
+                                              _ptr(tok_logprob), _stream()), "specs_merge_partials")
 
     def specs_prm_rewards(self, prm_hidden, block_offsets, w_head, bias, reward):
         """Value head of the PRM on each block's last hidden state, logistic link; reward float32 [B] out."""

@@ -303,6 +303,44 @@ int specs_score_blocks(specs_ctx* ctx, const void* hidden, const void* W_vocab, 
     return SPECS_OK;
 }
 
+int specs_score_partials(specs_ctx* ctx, const void* hidden, const void* W_shard, const int32_t* token_ids,
+                         int32_t id_offset, int64_t rows, int32_t d, int32_t V_shard, float* partials,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    int st = check_score_shapes(rows, d, V_shard, 0);
+    if (st != SPECS_OK) return st;
+    if (id_offset < 0) return SPECS_ERR_SHAPE;
+    if (rows == 0) return SPECS_OK;
+    if (!hidden || !W_shard || !token_ids || !partials || !workspace) return SPECS_ERR_NULL;
+    if (!aligned16(hidden) || !aligned16(W_shard) || !aligned16(workspace) || !aligned16(partials))
+        return SPECS_ERR_ALIGN;
+    if (ctx->engine == SPECS_ENGINE_SIMT) return SPECS_ERR_SHAPE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+    const int cta_group = ctx->engine == SPECS_ENGINE_TCGEN05_1CTA ? 1
+                        : ctx->engine == SPECS_ENGINE_TCGEN05_2CTA ? 2 : kCtaGroupAuto;
+    const ScorePlan plan = make_score_plan(rows, d, V_shard, ctx->num_sms, ctx->pair_units, cta_group,
+                                           ctx->chunk_kblocks, ctx->accum_adaptive);
+    if (workspace_bytes < plan_workspace_bytes(plan)) return SPECS_ERR_WORKSPACE;
+    st = launch_score_tcgen05(ctx, plan, hidden, W_shard, token_ids, static_cast<float*>(workspace), stream, id_offset);
+    if (st != SPECS_OK) return st;
+    return launch_row_partials(ctx, plan, static_cast<const float*>(workspace), partials, stream);
+}
+
+int specs_merge_partials(specs_ctx* ctx, const float* partials, int32_t shards, int64_t rows,
+                         const int32_t* token_ids, int32_t V, float* tok_logprob, void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    if (shards <= 0 || rows < 0 || V <= 0) return SPECS_ERR_SHAPE;
+    if (rows == 0) return SPECS_OK;
+    if (!partials || !token_ids || !tok_logprob) return SPECS_ERR_NULL;
+    if (!aligned16(partials)) return SPECS_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+    return launch_merge_partials(ctx, partials, shards, rows, token_ids, V, tok_logprob,
+                                 static_cast<cudaStream_t>(cuda_stream));
+}
+
 int specs_block_sums(specs_ctx* ctx, const float* per_token, const int64_t* block_offsets, int32_t B, float* out,
                      double* out_f64, void* cuda_stream) {
     if (!ctx) return SPECS_ERR_NULL;

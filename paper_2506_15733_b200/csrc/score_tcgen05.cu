@@ -640,7 +640,8 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
             int ck = plan.chunk_kblocks;                     // k-blocks per chunk of the current tile
             float assumed = INFINITY;                        // magnitude the lengthened chunks were sized for
             const int64_t row = (int64_t)(st * kCg + (int)rank) * kBlockM + row_in_tile;
-            const int32_t id = (row < plan.rows) ? token_ids[row] : -1;
+            // ids are indices into the whole vocabulary; this W holds rows id_offset .. id_offset + V - 1
+            const int32_t id = (row < plan.rows) ? token_ids[row] - plan.id_offset : -1;
             // state in base-2 units: run_max = max(z) * log2(e), run_sum = sum 2^(z*log2e - run_max)
             float run_max = -INFINITY, run_sum = 0.0f, picked = -INFINITY;
             for (int n = nb; n < ne && ok; ++n) {
@@ -836,7 +837,7 @@ int query_pair_units(int device, int num_sms) {
 }
 
 int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan_in, const void* hidden, const void* w_vocab,
-                         const int32_t* token_ids, float* workspace, cudaStream_t stream) {
+                         const int32_t* token_ids, float* workspace, cudaStream_t stream, int32_t id_offset) {
     static_assert(Shape<1>::kSmemBytes <= 227 * 1024 && Shape<2>::kSmemBytes <= 227 * 1024, "shared memory budget");
     static_assert(Shape<1>::kStages <= kMaxStages && Shape<2>::kStages <= kMaxStages, "barrier arrays");
     static_assert(sizeof(SharedLayout) <= 512, "barrier block");
@@ -846,6 +847,7 @@ int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan_in, const void* h
     ScorePlan plan = plan_in;
     plan.epoch = (launch_counter.fetch_add(1) % 0xfffeu) + 1u;  // never 0
     plan.lead_tiles = ctx->lead_tiles;
+    plan.id_offset = id_offset;
     query_pair_units(ctx->device, ctx->num_sms);             // shared-memory opt-in for this device
     CUtensorMap map_h, map_w;
     int st = encode_bf16_2d(ctx, &map_h, hidden, (uint64_t)plan.d, (uint64_t)plan.rows, kBlockK, kBlockM);

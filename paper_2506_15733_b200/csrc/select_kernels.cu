@@ -26,11 +26,12 @@ constexpr unsigned kFull = 0xffffffffu;
 // that saw no valid column (vocabulary tail) carries max = -inf, sum = 0.
 constexpr int kMergeBatch = 6;                              // splits whose six floats are loaded before any is used
 
-// log pi_target of the drafted token of `row`: fold the row's per-split partials, in split order,
-// into (max, sum) in base-2 units, then  logit - (max + log2 sum) * ln 2.  The loads of a batch of
-// splits are independent of the arithmetic and of each other, so a batch costs one trip to L2.
-__device__ __forceinline__ float merged_logprob(const ScorePlan& plan, const float* __restrict__ workspace,
-                                                int64_t row, int32_t id, uint32_t* __restrict__ status) {
+// Fold of a row's per-split partials, in split order, into (max, sum) in base-2 units and the drafted
+// id's logit.  The loads of a batch of splits are independent of the arithmetic and of each other, so a
+// batch costs one trip to L2.
+struct RowFold { float max2; double sum2; float logit; };
+
+__device__ __forceinline__ RowFold fold_row(const ScorePlan& plan, const float* __restrict__ workspace, int64_t row) {
     const int mt = (int)(row / kBlockM), r = (int)(row % kBlockM);
     // the row tile's work unit: super tile (cta_group row tiles) and the CTA's rank inside the unit
     const int cg = plan.cta_group, sup = mt / cg, rank = mt % cg;
@@ -45,8 +46,8 @@ __device__ __forceinline__ float merged_logprob(const ScorePlan& plan, const flo
     const size_t stride = (size_t)gm * cg * kTripleFloats;  // next chunk of the same row tile
     constexpr int kHalf = 3 * kBlockM;                      // second half of the tile's columns
 
-    float m = -INFINITY, logit = -INFINITY;
-    double sum = 0.0;
+    RowFold f;
+    f.max2 = -INFINITY; f.sum2 = 0.0; f.logit = -INFINITY;
     for (int s0 = 0; s0 < splits; s0 += kMergeBatch) {
         float v[kMergeBatch][6];
 #pragma unroll
@@ -60,22 +61,66 @@ __device__ __forceinline__ float merged_logprob(const ScorePlan& plan, const flo
         }
 #pragma unroll
         for (int u = 0; u < kMergeBatch; ++u) {
-            const float mn = fmaxf(m, fmaxf(v[u][0], v[u][3]));
+            const float mn = fmaxf(f.max2, fmaxf(v[u][0], v[u][3]));
             if (mn != -INFINITY) {
                 // exp2f(-inf) = 0 takes care of halves and states that have seen nothing yet
-                sum = sum * (double)exp2f(m - mn) + (double)v[u][1] * (double)exp2f(v[u][0] - mn) +
-                      (double)v[u][4] * (double)exp2f(v[u][3] - mn);
-                m = mn;
+                f.sum2 = f.sum2 * (double)exp2f(f.max2 - mn) + (double)v[u][1] * (double)exp2f(v[u][0] - mn) +
+                         (double)v[u][4] * (double)exp2f(v[u][3] - mn);
+                f.max2 = mn;
             }
-            logit = fmaxf(logit, fmaxf(v[u][2], v[u][5]));
+            f.logit = fmaxf(f.logit, fmaxf(v[u][2], v[u][5]));
         }
     }
+    return f;
+}
+
+// log pi_target of the drafted token of `row`:  logit - (max + log2 sum) * ln 2.
+__device__ __forceinline__ float merged_logprob(const ScorePlan& plan, const float* __restrict__ workspace,
+                                                int64_t row, int32_t id, uint32_t* __restrict__ status) {
+    const RowFold f = fold_row(plan, workspace, row);
     if (id < 0 || id >= plan.V) {
         atomicOr(status, SPECS_DEV_TOKEN_RANGE);
         return __int_as_float(0x7fc00000);                  // no such vocabulary entry: NaN
     }
-    const double lse = ((double)m + log2(sum)) * kLn2;      // natural-log normaliser
-    return (float)((double)logit - lse);
+    const double lse = ((double)f.max2 + log2(f.sum2)) * kLn2;   // natural-log normaliser
+    return (float)((double)f.logit - lse);
+}
+
+// One row's fold as it stands, for a holder of one shard of the vocabulary: partials[row] =
+// (max in base-2 units, sum of 2^(x - max), drafted id's logit or -inf, 0).
+__global__ void __launch_bounds__(128)
+row_partials_kernel(const ScorePlan plan, const float* __restrict__ workspace, float4* __restrict__ partials) {
+    const int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= plan.rows) return;
+    const RowFold f = fold_row(plan, workspace, row);
+    partials[row] = make_float4(f.max2, (float)f.sum2, f.logit, 0.0f);
+}
+
+// The same fold over the shards' partials [shards, rows]: log pi_target of the drafted id.
+__global__ void __launch_bounds__(128)
+merge_partials_kernel(const float4* __restrict__ partials, int32_t shards, int64_t rows,
+                      const int32_t* __restrict__ token_ids, int32_t V, float* __restrict__ tok_logprob,
+                      uint32_t* __restrict__ status) {
+    const int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= rows) return;
+    float m = -INFINITY, logit = -INFINITY;
+    double sum = 0.0;
+    for (int j = 0; j < shards; ++j) {
+        const float4 v = partials[(size_t)j * rows + row];
+        const float mn = fmaxf(m, v.x);
+        if (mn != -INFINITY) {
+            sum = sum * (double)exp2f(m - mn) + (double)v.y * (double)exp2f(v.x - mn);
+            m = mn;
+        }
+        logit = fmaxf(logit, v.z);
+    }
+    const int32_t id = token_ids[row];
+    if (id < 0 || id >= V) {
+        tok_logprob[row] = __int_as_float(0x7fc00000);
+        atomicOr(status, SPECS_DEV_TOKEN_RANGE);
+        return;
+    }
+    tok_logprob[row] = (float)((double)logit - ((double)m + log2(sum)) * kLn2);
 }
 
 __global__ void __launch_bounds__(128)
@@ -430,6 +475,23 @@ int launch_gather_chosen(const int32_t* token_ids, const int64_t* block_offsets,
     if (P == 0) return SPECS_OK;
     gather_chosen_kernel<<<(unsigned)P, 128, 0, stream>>>(token_ids, block_offsets, cand_offsets, chosen, chosen_ids,
                                                           chosen_len, stride);
+    return cuda_status(cudaGetLastError());
+}
+
+int launch_row_partials(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, float* partials,
+                        cudaStream_t stream) {
+    (void)ctx;
+    if (plan.rows == 0) return SPECS_OK;
+    row_partials_kernel<<<(unsigned)((plan.rows + 127) / 128), 128, 0, stream>>>(plan, workspace,
+                                                                               reinterpret_cast<float4*>(partials));
+    return cuda_status(cudaGetLastError());
+}
+
+int launch_merge_partials(specs_ctx* ctx, const float* partials, int32_t shards, int64_t rows, const int32_t* token_ids,
+                          int32_t V, float* tok_logprob, cudaStream_t stream) {
+    if (rows == 0) return SPECS_OK;
+    merge_partials_kernel<<<(unsigned)((rows + 127) / 128), 128, 0, stream>>>(
+        reinterpret_cast<const float4*>(partials), shards, rows, token_ids, V, tok_logprob, ctx->d_status);
     return cuda_status(cudaGetLastError());
 }
 

@@ -53,6 +53,7 @@ struct ScorePlan {
     int32_t chunk_kblocks; // k-blocks per fresh tensor-core accumulator (chunks are summed in registers)
     int32_t lead_tiles;    // > 0: a unit starts vocabulary tile t of a wave only once every unit that streams the
                            //      same W chunk has started tile t - lead_tiles (advisory, bounded wait)
+    int32_t id_offset;     // vocabulary index of W_vocab's first row (a shard of a larger vocabulary); 0 normally
     uint32_t epoch;        // distinguishes this launch's progress words from older contents of the workspace
     int32_t adaptive;      // 1: from the third vocabulary tile of a run on, lengthen the chunks as far as the
                            //    logit magnitude seen in the run's first tile allows (see score_tcgen05.cu)
@@ -121,7 +122,7 @@ namespace specs {
 // device; also opts both kernels in to their dynamic shared memory).  0 if pairs cannot launch.
 int query_pair_units(int device, int num_sms);
 int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan, const void* hidden, const void* w_vocab,
-                         const int32_t* token_ids, float* workspace, cudaStream_t stream);
+                         const int32_t* token_ids, float* workspace, cudaStream_t stream, int32_t id_offset = 0);
 int launch_score_simt(specs_ctx* ctx, const void* hidden, const void* w_vocab, const int32_t* token_ids,
                       int64_t rows, int32_t d, int32_t V, float* tok_logprob, cudaStream_t stream);
 int launch_merge(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, const int32_t* token_ids,
@@ -135,6 +136,10 @@ int launch_finish_step(specs_ctx* ctx, const ScorePlan& plan, const float* works
 int launch_gather_chosen(const int32_t* token_ids, const int64_t* block_offsets, const int32_t* cand_offsets,
                          const int32_t* chosen, int32_t P, int32_t* chosen_ids, int32_t* chosen_len, int32_t stride,
                          cudaStream_t stream);
+int launch_row_partials(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, float* partials,
+                        cudaStream_t stream);
+int launch_merge_partials(specs_ctx* ctx, const float* partials, int32_t shards, int64_t rows, const int32_t* token_ids,
+                          int32_t V, float* tok_logprob, cudaStream_t stream);
 int launch_block_sums(const float* per_token, const int64_t* block_offsets, int32_t B,
                       float* out, double* out_f64, cudaStream_t stream);
 int launch_subsample(const void* lp_target, const void* lp_gen, bool lp_is_f64, const float* reward,

@@ -636,3 +636,52 @@ def test_prm_head_matches_the_oracle_and_overlaps_with_scoring(ctx):
         ctx.specs_prm_rewards(s.hidden[:, :12], s.block_offsets, w_dev, 0.0, reward)
     assert e.value.status == 2
     assert ctx.device_status() == 0
+
+
+# ------------------------------------------------------------------------------- vocabulary shards
+
+@pytest.mark.parametrize("world", [1, 3])
+def test_vocab_sharded_scoring_matches_oracle_and_single_gpu_path(ctx, world):
+    # the ranks' kernels emulated one after the other on this GPU; the exchange itself is tested under gloo
+    from paper_2506_15733_b200 import vocab_parallel as VP
+    cfg = small_config("shards", (5, 40), 2, 5, 192, 5000, seed=5800)      # 19.5 vocabulary tiles: ragged last shard
+    x = I.make_step_inputs(cfg)
+    x.token_ids = x.token_ids.copy()
+    x.token_ids[7] = 5000                                                   # not in any shard
+    dev = "cuda:0"
+    s = DeviceStep(ctx, x)
+    parts, bounds = [], []
+    for rank in range(world):
+        v0, v1 = VP.shard_bounds(5000, world, rank)
+        bounds.append((v0, v1))
+        w_shard = s.w_vocab[v0:v1]
+        local = torch.full((x.rows, 4), float("nan"), dtype=torch.float32, device=dev)
+        ws = torch.empty(ctx.score_workspace_bytes(x.rows, 192, v1 - v0), dtype=torch.uint8, device=dev)
+        ctx.specs_score_partials(s.hidden, w_shard, s.token_ids, v0, local, ws)
+        parts.append(local)
+    assert bounds[0][0] == 0 and bounds[-1][1] == 5000 and all(a[1] == b[0] for a, b in zip(bounds, bounds[1:]))
+    allp = torch.stack(parts)
+    out = torch.full((x.rows,), 7.0, dtype=torch.float32, device=dev)
+    ctx.specs_merge_partials(allp, s.token_ids, 5000, out)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    want = O.token_logprobs(x.hidden, x.w_vocab, x.token_ids)
+    assert np.isnan(got[7]) and np.isnan(want[7])
+    ok = np.arange(x.rows) != 7
+    assert np.abs(got[ok] - want[ok]).max() <= TOK_ATOL
+    assert ctx.device_status() == binding.DEV_TOKEN_RANGE
+    # each shard's partials against the oracle's (natural units there, base-2 units here)
+    p_np = allp.cpu().numpy().astype(np.float64)
+    for rank, (v0, v1) in enumerate(bounds):
+        ref = OV.shard_partials(x.hidden, x.w_vocab, x.token_ids, v0, v1)
+        lse_ref = ref[:, 0] + np.log(ref[:, 1])
+        lse_got = (p_np[rank, :, 0] + np.log2(p_np[rank, :, 1])) * math.log(2.0)
+        assert np.abs(lse_got - lse_ref).max() <= TOK_ATOL
+        held = np.isfinite(ref[:, 2])
+        assert np.array_equal(np.isfinite(p_np[rank, :, 2]), held)
+        assert np.abs(p_np[rank, held, 2] - ref[held, 2]).max() <= TOK_ATOL
+    # and the unsharded path
+    s.score()
+    torch.cuda.synchronize()
+    assert np.abs(s.tok_lp.cpu().numpy()[ok] - got[ok]).max() <= 1e-5
+    ctx.device_status()
