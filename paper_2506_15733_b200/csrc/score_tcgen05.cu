@@ -8,7 +8,10 @@
 //
 // Persistent CTAs, one per SM, 384 threads (three warpgroups), three roles:
 //   warp 0      TMA producer: cp.async.bulk.tensor loads of a 128x64 hidden tile and a W tile
-//               per k-block into a ring of 128-byte-swizzled shared-memory stages.
+//               per k-block into a ring of 128-byte-swizzled shared-memory stages (lane 0).
+//               Before each vocabulary tile the warp paces itself against the other units
+//               that stream the same W chunk (see "pacing" below), so that a W tile is
+//               fetched from HBM once and found in L2 by the rest.
 //   warp 1      MMA issuer: one thread issues tcgen05.mma (N=256, K=16, bf16 -> fp32) into one
 //               of two 128-lane x 256-column TMEM buffers.  The reduction over d is cut into
 //               chunks of plan.chunk_kblocks k-blocks; every chunk starts a fresh accumulator
@@ -54,10 +57,6 @@
 #include <atomic>
 
 #include "specs_internal.h"
-
-#ifndef SPECS_TMA_HINTS
-#define SPECS_TMA_HINTS 0
-#endif
 
 namespace specs {
 namespace {
@@ -203,33 +202,6 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
         "[%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c_inner), "r"(c_outer), "r"(cluster_bar)
-        : "memory");
-}
-// L2 eviction-priority policies for the two operand streams.
-__device__ __forceinline__ uint64_t l2_policy_evict_last() {
-    uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
-    return p;
-}
-__device__ __forceinline__ uint64_t l2_policy_evict_first() {
-    uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-    return p;
-}
-__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer,
-                                                 uint32_t bar, uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
-        "[%0], [%1, {%2, %3}], [%4], %5;"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c_inner), "r"(c_outer), "r"(bar), "l"(policy)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_2d_pair_hint(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer,
-                                                      uint32_t cluster_bar, uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
-        "[%0], [%1, {%2, %3}], [%4], %5;"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c_inner), "r"(c_outer), "r"(cluster_bar), "l"(policy)
         : "memory");
 }
 // 2^x on the special-function unit (relative error about 2^-22; 2^-inf = 0).
@@ -449,13 +421,6 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
         // poll before each vocabulary tile (one progress word per lane, one trip to L2).
         // pair: every load of either CTA is counted on the leader's barrier of the stage
         const uint32_t full0 = (kCg == 2) ? mapa_shared(smem_u32(&sh->full[0]), 0u) : smem_u32(&sh->full[0]);
-#if SPECS_TMA_HINTS == 1
-        const uint64_t pol_h = l2_policy_evict_last(), pol_w = l2_policy_evict_first();
-#elif SPECS_TMA_HINTS == 2
-        const uint64_t pol_h = l2_policy_evict_last(), pol_w = l2_policy_evict_last();
-#elif SPECS_TMA_HINTS == 3
-        const uint64_t pol_h = l2_policy_evict_first(), pol_w = l2_policy_evict_last();
-#endif
         unsigned long long* progress = reinterpret_cast<unsigned long long*>(
             reinterpret_cast<char*>(workspace) + plan_slot_bytes(plan));
         bool pace = plan.lead_tiles > 0 && rank == 0;
@@ -515,13 +480,8 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                         } else {
                             // the leader expects both CTAs' bytes; the peer's may be counted first
                             if (rank == 0) mbar_arrive_expect_tx(smem_u32(&sh->full[stage]), 2u * kStageBytes);
-#if SPECS_TMA_HINTS
-                            tma_load_2d_pair_hint(a_dst, &map_hidden, kb * kBlockK, row0, bar, pol_h);
-                            tma_load_2d_pair_hint(a_dst + kABytes, &map_w, kb * kBlockK, wrow0, bar, pol_w);
-#else
                             tma_load_2d_pair(a_dst, &map_hidden, kb * kBlockK, row0, bar);
                             tma_load_2d_pair(a_dst + kABytes, &map_w, kb * kBlockK, wrow0, bar);
-#endif
                         }
                         ++issued;
                         if (++stage == kStages) { stage = 0; phase ^= 1u; }
