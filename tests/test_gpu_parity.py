@@ -685,3 +685,33 @@ def test_vocab_sharded_scoring_matches_oracle_and_single_gpu_path(ctx, world):
     torch.cuda.synchronize()
     assert np.abs(s.tok_lp.cpu().numpy()[ok] - got[ok]).max() <= 1e-5
     ctx.device_status()
+
+
+# ------------------------------------------------------------------------------- pacing is advisory
+
+@pytest.mark.parametrize("lead", [0, 1, 3])
+def test_pacing_never_changes_results_even_on_a_garbage_workspace(ctx, lead):
+    # several waves and several units per vocabulary chunk, so that the pacing path really runs; the workspace
+    # starts as random bytes (progress words of "another launch", some looking far ahead): only time may be lost
+    cfg = small_config("pace", (250, 250), 4, 10, 128, 2600, seed=5900, w_sigma=0.1)
+    x = I.make_step_inputs(cfg)
+    plan = binding.score_plan(x.rows, 128, 2600, ctx.sm_count())
+    assert plan["waves"] >= 2 and plan["group_m"] > 1
+    want = O.token_logprobs(x.hidden, x.w_vocab, x.token_ids)
+    s = DeviceStep(ctx, x)
+    ctx.set_tile_lead(lead)
+    try:
+        for fill in ("random", "ones"):
+            if fill == "random":
+                g = torch.Generator(device="cuda:0"); g.manual_seed(5901)
+                s.workspace.copy_(torch.randint(0, 256, s.workspace.shape, generator=g, device="cuda:0",
+                                                dtype=torch.uint8))
+            else:
+                s.workspace.fill_(0xff)
+            s.tok_lp.fill_(float("nan"))
+            s.score()
+            torch.cuda.synchronize()
+            assert np.abs(s.tok_lp.cpu().numpy() - want).max() <= TOK_ATOL
+    finally:
+        ctx.set_tile_lead(1)
+    assert ctx.device_status() == 0
