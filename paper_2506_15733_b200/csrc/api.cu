@@ -191,6 +191,7 @@ int specs_destroy(specs_ctx* ctx) {
     DeviceGuard guard(ctx->device);
     for (auto& t : ctx->timed) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
     if (ctx->arena) cudaFree(ctx->arena);
+    if (ctx->h_stage) cudaFreeHost(ctx->h_stage);
     if (ctx->d_status) cudaFree(ctx->d_status);
     delete ctx;
     return SPECS_OK;
@@ -592,14 +593,20 @@ int specs_beam_step_host(specs_ctx* ctx, const void* h_hidden, const void* W_voc
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return SPECS_ERR_CUDA;
 
-    // carve the arena (every piece 256-byte aligned)
+    // Carve the arena (every piece 256-byte aligned): hidden states, then one block of the small inputs, then
+    // one block of the outputs, then what never crosses the bus.  The two blocks are mirrored in a pinned
+    // staging buffer so that each crosses in ONE copy instead of one copy per array.
     size_t off = 0;
     auto carve = [&off](size_t bytes) { const size_t at = off; off += (bytes + 255) & ~(size_t)255; return at; };
-    const size_t o_hidden = carve((size_t)rows * d * 2), o_ids = carve((size_t)rows * 4);
-    const size_t o_boff = carve((size_t)(B + 1) * 8), o_coff = carve((size_t)(P + 1) * 4);
+    const size_t o_hidden = carve((size_t)rows * d * 2);
+    const size_t in0 = off;
+    const size_t o_ids = carve((size_t)rows * 4), o_boff = carve((size_t)(B + 1) * 8), o_coff = carve((size_t)(P + 1) * 4);
     const size_t o_gen = carve((size_t)rows * 4), o_rew = carve((size_t)B * 4), o_uni = carve((size_t)B * 4);
-    const size_t o_tok = carve((size_t)rows * 4), o_blk_t = carve((size_t)B * 8), o_blk_g = carve((size_t)B * 8);
-    const size_t o_wts = carve((size_t)B * 4), o_cho = carve((size_t)P * 4), o_acc = carve((size_t)P);
+    const size_t out0 = off;
+    const size_t o_tok = carve((size_t)rows * 4), o_blk_t = carve((size_t)B * 8), o_wts = carve((size_t)B * 4);
+    const size_t o_cho = carve((size_t)P * 4), o_acc = carve((size_t)P);
+    const size_t out1 = off;
+    const size_t o_blk_g = carve((size_t)B * 8);
     const size_t ws_bytes = specs_score_workspace_bytes(ctx, rows, d, V);
     const size_t o_ws = carve(ws_bytes);
     if (off > ctx->arena_bytes) {
@@ -607,18 +614,26 @@ int specs_beam_step_host(specs_ctx* ctx, const void* h_hidden, const void* W_voc
         if (cudaMalloc(&ctx->arena, off) != cudaSuccess) return SPECS_ERR_CUDA;
         ctx->arena_bytes = off;
     }
+    const size_t stage_bytes = out1 - in0;
+    if (stage_bytes > ctx->stage_bytes) {
+        if (ctx->h_stage) { cudaStreamSynchronize(stream); cudaFreeHost(ctx->h_stage); ctx->h_stage = nullptr; ctx->stage_bytes = 0; }
+        if (cudaMallocHost(&ctx->h_stage, stage_bytes) != cudaSuccess) return SPECS_ERR_CUDA;
+        ctx->stage_bytes = stage_bytes;
+    }
     uint8_t* A = static_cast<uint8_t*>(ctx->arena);
-    auto h2d = [&](size_t at, const void* src, size_t bytes) {
-        return bytes == 0 || cudaMemcpyAsync(A + at, src, bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
-    };
-    auto d2h = [&](void* dst, size_t at, size_t bytes) {
-        return !dst || bytes == 0 || cudaMemcpyAsync(dst, A + at, bytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
-    };
-    bool ok = h2d(o_hidden, h_hidden, (size_t)rows * d * 2) && h2d(o_ids, h_token_ids, (size_t)rows * 4) &&
-              h2d(o_boff, h_block_offsets, (size_t)(B + 1) * 8) && h2d(o_coff, h_cand_offsets, (size_t)(P + 1) * 4) &&
-              h2d(o_rew, h_reward, (size_t)B * 4) && h2d(o_uni, h_uniforms, (size_t)B * 4);
-    if (ok && h_gen_tok_logprob) ok = h2d(o_gen, h_gen_tok_logprob, (size_t)rows * 4);
-    if (!ok) return SPECS_ERR_CUDA;
+    uint8_t* S = static_cast<uint8_t*>(ctx->h_stage) - in0;          // S + offset mirrors A + offset
+    auto put = [&](size_t at, const void* src, size_t bytes) { if (src && bytes) std::memcpy(S + at, src, bytes); };
+    put(o_ids, h_token_ids, (size_t)rows * 4);
+    put(o_boff, h_block_offsets, (size_t)(B + 1) * 8);
+    put(o_coff, h_cand_offsets, (size_t)(P + 1) * 4);
+    put(o_gen, h_gen_tok_logprob, (size_t)rows * 4);
+    put(o_rew, h_reward, (size_t)B * 4);
+    put(o_uni, h_uniforms, (size_t)B * 4);
+    if (rows > 0 && cudaMemcpyAsync(A + o_hidden, h_hidden, (size_t)rows * d * 2, cudaMemcpyHostToDevice, stream) !=
+                        cudaSuccess)
+        return SPECS_ERR_CUDA;
+    if (cudaMemcpyAsync(A + in0, S + in0, out0 - in0, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return SPECS_ERR_CUDA;
 
     st = specs_beam_step(ctx, A + o_hidden, W_vocab, reinterpret_cast<int32_t*>(A + o_ids),
                          reinterpret_cast<int64_t*>(A + o_boff), reinterpret_cast<int32_t*>(A + o_coff),
@@ -629,10 +644,15 @@ int specs_beam_step_host(specs_ctx* ctx, const void* h_hidden, const void* W_voc
                          reinterpret_cast<int32_t*>(A + o_cho), reinterpret_cast<uint8_t*>(A + o_acc), A + o_ws,
                          ws_bytes, cuda_stream);
     if (st != SPECS_OK) return st;
-    ok = d2h(h_tok_logprob, o_tok, (size_t)rows * 4) && d2h(h_blk_logprob, o_blk_t, (size_t)B * 8) &&
-         d2h(h_weights, o_wts, (size_t)B * 4) && d2h(h_chosen, o_cho, (size_t)P * 4) &&
-         d2h(h_accept, o_acc, (size_t)P);
-    if (!ok || cudaStreamSynchronize(stream) != cudaSuccess) return SPECS_ERR_CUDA;
+    if (cudaMemcpyAsync(S + out0, A + out0, out1 - out0, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess)
+        return SPECS_ERR_CUDA;
+    auto get = [&](void* dst, size_t at, size_t bytes) { if (dst && bytes) std::memcpy(dst, S + at, bytes); };
+    get(h_tok_logprob, o_tok, (size_t)rows * 4);
+    get(h_blk_logprob, o_blk_t, (size_t)B * 8);
+    get(h_weights, o_wts, (size_t)B * 4);
+    get(h_chosen, o_cho, (size_t)P * 4);
+    get(h_accept, o_acc, (size_t)P);
     return SPECS_OK;
 }
 

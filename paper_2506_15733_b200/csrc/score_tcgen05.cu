@@ -55,6 +55,7 @@
 #include <cuda_bf16.h>
 
 #include <atomic>
+#include <mutex>
 
 #include "specs_internal.h"
 
@@ -768,6 +769,8 @@ int query_pair_units(int device, int num_sms) {
     // attribute) and ask how many CTA pairs the device keeps resident at once.
     static int cached[64];
     static bool done[64] = {};
+    static std::mutex guard;
+    std::lock_guard<std::mutex> lock(guard);
     const int slot = device & 63;
     if (done[slot]) return cached[slot];
     int units = 0;

@@ -109,6 +109,8 @@ struct specs_ctx {
     // grow-only device arena for specs_beam_step_host
     void* arena = nullptr;
     size_t arena_bytes = 0;
+    void* h_stage = nullptr;               // pinned mirror of the arena's small-input and output blocks
+    size_t stage_bytes = 0;
     // optional per-launch timing of the tensor-core kernel
     bool timing = false;
     std::vector<specs::TimedLaunch> timed;
