@@ -195,6 +195,22 @@ def test_dual_head_step_at_full_size(ctx):
     assert np.array_equal(ids_out.cpu().numpy(), want_ids) and np.array_equal(len_out.cpu().numpy(), want_len)
 
 
+@pytest.mark.parametrize("d", [2048, 4096])
+def test_llama_shaped_heads(ctx, d):
+    # the paper's second model pair (Llama-3.2-1B / Llama-3.1-8B, Section 4.1): d = 2048 / 4096, V = 128256
+    cfg = I.StepConfig(f"llama_{d}", 1100 + d, 2, 8, (48, 96), d, 128256, 0.02, reward_dist=("beta", 2.0, 2.0),
+                       betas=(1.0,))
+    x = I.make_step_inputs(cfg)
+    s = DeviceStep(ctx, x)
+    got = s.step(1.0, 0.7)
+    rng = np.random.Generator(np.random.Philox(key=[7006, d]))
+    blocks = sorted(rng.choice(x.blocks, size=2, replace=False).tolist())
+    rows_idx = np.unique(np.concatenate([rows_of_blocks(x, blocks), rng.choice(x.rows, 64, replace=False)]))
+    want_tok, err = check_sampled_rows(x, got["tok_logprob"], rows_idx, O.bf16_bits_to_f64(x.w_vocab))
+    check_block_sums(x, got, blocks, dict(zip(rows_idx.tolist(), want_tok.tolist())))
+    check_selection_logic(x, got, 1.0, 0.7, O.block_sums(x.draft_tok_logprob, x.block_offsets))
+
+
 def test_stress_heavy_tailed_logits(ctx):
     cfg = I.CONFIGS["stress"]
     x = I.make_step_inputs(cfg)
