@@ -174,6 +174,8 @@ def main():
     ap.add_argument("--oracle-blocks", type=int, default=16, help="whole blocks per CPU-oracle sample")
     ap.add_argument("--tile-lead", type=int, default=None,
                     help="pacing of the CTA pairs that stream the same W chunk, in vocabulary tiles (0: off; default: the library's)")
+    ap.add_argument("--time-every", type=int, default=1,
+                    help="record CUDA events around the scoring kernel on every K-th step of the timed region")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -236,13 +238,18 @@ def main():
     for _ in range(args.warmup):
         step()
     barrier()
-    ctx.set_timing(True)
+    every = max(1, args.time_every)
+    ctx.set_timing(every == 1)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(physical_gpu_index(local_rank)) as clocks:
         barrier()
         e0.record()
-        for _ in range(args.steps):
+        for k in range(args.steps):
+            if every > 1 and k % every == 0:
+                ctx.resume_timing()
             step()
+            if every > 1 and k % every == 0:
+                ctx.pause_timing()
         e1.record()
         barrier()
     total_ms = e0.elapsed_time(e1)

@@ -404,12 +404,14 @@ int specs_beam_step_host(specs_ctx* ctx,
                          int32_t* h_chosen, uint8_t* h_accept, void* cuda_stream);
 
 /* Per-launch timing of the tensor-core scoring kernel.  specs_set_timing(ctx, 1)
- * makes every later specs_score_blocks call on this context record a CUDA event
- * before and after that kernel on the call's own stream (a few microseconds each;
- * off by default) and forgets earlier records; specs_set_timing(ctx, 0) stops.
- * specs_score_kernel_ms() waits for the recorded launches, returns their MEAN
- * duration in milliseconds, stores their number in *h_launches (may be NULL) and
- * forgets them; it returns a negative value when nothing was recorded. */
+ * makes every later scoring call on this context record a CUDA event before and
+ * after that kernel on the call's own stream (a few microseconds each; off by
+ * default) and forgets earlier records; (ctx, 0) stops recording and keeps the
+ * records; (ctx, 2) resumes recording without forgetting, so that a caller can
+ * time every K-th launch of a loop.  specs_score_kernel_ms() waits for the recorded
+ * launches, returns their MEAN duration in milliseconds, stores their number in
+ * *h_launches (may be NULL) and forgets them; it returns a negative value when
+ * nothing was recorded. */
 int   specs_set_timing(specs_ctx* ctx, int enabled);
 float specs_score_kernel_ms(specs_ctx* ctx, int32_t* h_launches);
 

@@ -182,6 +182,12 @@ class Context:
     def set_timing(self, enabled: bool):
         _check(self._lib.specs_set_timing(self._h, 1 if enabled else 0), "specs_set_timing")
 
+    def pause_timing(self):
+        _check(self._lib.specs_set_timing(self._h, 0), "specs_set_timing")
+
+    def resume_timing(self):
+        _check(self._lib.specs_set_timing(self._h, 2), "specs_set_timing")
+
     def score_kernel_ms(self):
         n = _i32(0)
         ms = float(self._lib.specs_score_kernel_ms(self._h, C.byref(n)))

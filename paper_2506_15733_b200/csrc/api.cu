@@ -550,8 +550,9 @@ int specs_device_status(specs_ctx* ctx, uint32_t* h_bits, void* cuda_stream) {
 
 int specs_set_timing(specs_ctx* ctx, int enabled) {
     if (!ctx) return SPECS_ERR_NULL;
+    if (enabled < 0 || enabled > 2) return SPECS_ERR_SHAPE;
     ctx->timing = enabled != 0;
-    ctx->timed_used = 0;
+    if (enabled == 1) ctx->timed_used = 0;                   // a fresh start forgets earlier records
     return SPECS_OK;
 }
 
