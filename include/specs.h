@@ -403,6 +403,15 @@ int specs_beam_step_host(specs_ctx* ctx,
                          float* h_tok_logprob, double* h_blk_logprob, float* h_weights,
                          int32_t* h_chosen, uint8_t* h_accept, void* cuda_stream);
 
+/* Failure-detection self-test.  Every wait inside the scoring kernel is bounded: when
+ * its time runs out it raises SPECS_DEV_TIMEOUT in the device status word and the
+ * kernel winds down instead of hanging.  This call launches a one-CTA kernel that
+ * runs that same wait, for limit_us microseconds (1 .. 1 000 000), on a barrier that
+ * nothing completes: afterwards specs_device_status() must report
+ * SPECS_ERR_DEVICE_TIMEOUT, and the context must remain usable.  (The paper has no
+ * counterpart; it is how the expiry path is tested without a stuck GPU.) */
+int specs_probe_wait_expiry(specs_ctx* ctx, int64_t limit_us, void* cuda_stream);
+
 /* Per-launch timing of the tensor-core scoring kernel.  specs_set_timing(ctx, 1)
  * makes every later scoring call on this context record a CUDA event before and
  * after that kernel on the call's own stream (a few microseconds each; off by

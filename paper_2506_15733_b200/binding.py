@@ -70,6 +70,7 @@ SIGNATURES = {
     "specs_device_status": (C.c_int, [_vp, C.POINTER(C.c_uint32), _vp]),
     "specs_beam_step_host": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32,
                                        _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "specs_probe_wait_expiry": (C.c_int, [_vp, _i64, _vp]),
     "specs_set_timing": (C.c_int, [_vp, C.c_int]),
     "specs_score_kernel_ms": (C.c_float, [_vp, C.POINTER(_i32)]),
     "specs_score_blocks_noalloc": (C.c_int, [_vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]),
@@ -178,6 +179,9 @@ class Context:
 
     def score_workspace_bytes(self, rows: int, d: int, V: int) -> int:
         return int(self._lib.specs_score_workspace_bytes(self._h, rows, d, V))
+
+    def probe_wait_expiry(self, limit_us: int):
+        _check(self._lib.specs_probe_wait_expiry(self._h, int(limit_us), _stream()), "specs_probe_wait_expiry")
 
     def set_timing(self, enabled: bool):
         _check(self._lib.specs_set_timing(self._h, 1 if enabled else 0), "specs_set_timing")

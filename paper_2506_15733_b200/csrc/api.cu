@@ -548,6 +548,14 @@ int specs_device_status(specs_ctx* ctx, uint32_t* h_bits, void* cuda_stream) {
     return SPECS_OK;
 }
 
+int specs_probe_wait_expiry(specs_ctx* ctx, int64_t limit_us, void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    if (limit_us <= 0 || limit_us > 1000000) return SPECS_ERR_SHAPE;   // at most one second
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+    return launch_wait_expiry_probe(ctx, (unsigned long long)limit_us * 1000ull, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int specs_set_timing(specs_ctx* ctx, int enabled) {
     if (!ctx) return SPECS_ERR_NULL;
     if (enabled < 0 || enabled > 2) return SPECS_ERR_SHAPE;

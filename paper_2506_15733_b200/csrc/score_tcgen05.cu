@@ -749,6 +749,27 @@ score_tiles_pair_kernel(const __grid_constant__ CUtensorMap map_hidden, const __
     score_tiles_body<2>(map_hidden, map_w, plan, token_ids, workspace, status);
 }
 
+// One CTA waits, with the kernel's own bounded wait, on a barrier that nothing ever completes:
+// the wait must give up after limit_ns, raise the abort flag and report SPECS_DEV_TIMEOUT, and
+// the kernel must return.  This is the expiry path of every wait in the scoring kernel,
+// exercised without a stuck scoring kernel.
+__global__ void wait_expiry_probe_kernel(unsigned long long limit_ns, uint32_t* __restrict__ status) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    AbortFlags ab;
+    ab.own = &abort_flag;
+    ab.peer = 0u;
+    const bool completed = mbar_wait(smem_u32(&bar), 0u, ab, limit_ns, true);
+    __syncthreads();
+    if (threadIdx.x == 0 && (!completed || abort_flag != 0u)) atomicOr(status, SPECS_DEV_TIMEOUT);
+}
+
 int encode_bf16_2d(specs_ctx* ctx, CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer,
                    uint32_t box_inner, uint32_t box_outer) {
     const cuuint64_t dims[2] = {inner, outer};
@@ -763,6 +784,11 @@ int encode_bf16_2d(specs_ctx* ctx, CUtensorMap* map, const void* base, uint64_t 
 }
 
 }  // namespace
+
+int launch_wait_expiry_probe(specs_ctx* ctx, unsigned long long limit_ns, cudaStream_t stream) {
+    wait_expiry_probe_kernel<<<1, 64, 0, stream>>>(limit_ns, ctx->d_status);
+    return cuda_status(cudaGetLastError());
+}
 
 int query_pair_units(int device, int num_sms) {
     // Per device, once: opt both kernels in to their dynamic shared memory (a per-device function

@@ -125,6 +125,7 @@ namespace specs {
 int query_pair_units(int device, int num_sms);
 int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan, const void* hidden, const void* w_vocab,
                          const int32_t* token_ids, float* workspace, cudaStream_t stream, int32_t id_offset = 0);
+int launch_wait_expiry_probe(specs_ctx* ctx, unsigned long long limit_ns, cudaStream_t stream);
 int launch_score_simt(specs_ctx* ctx, const void* hidden, const void* w_vocab, const int32_t* token_ids,
                       int64_t rows, int32_t d, int32_t V, float* tok_logprob, cudaStream_t stream);
 int launch_merge(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, const int32_t* token_ids,

@@ -715,3 +715,24 @@ def test_pacing_never_changes_results_even_on_a_garbage_workspace(ctx, lead):
     finally:
         ctx.set_tile_lead(1)
     assert ctx.device_status() == 0
+
+
+# ------------------------------------------------------------------------------- bounded waits
+
+def test_a_wait_that_nothing_completes_expires_and_is_reported(ctx):
+    import time
+    t0 = time.perf_counter()
+    ctx.probe_wait_expiry(2000)                                   # 2 ms on a barrier nobody arrives at
+    with pytest.raises(binding.SpecsError) as e:
+        ctx.device_status(raise_on_error=True)                    # synchronises: the kernel did return
+    assert e.value.status == 8                                    # SPECS_ERR_DEVICE_TIMEOUT
+    assert time.perf_counter() - t0 < 5.0
+    assert ctx.device_status() == 0                               # reading cleared the word
+    # the context is as usable as before
+    x = I.make_step_inputs(I.CONFIGS["tiny"])
+    got = DeviceStep(ctx, x).step(1.0, 0.7)
+    assert_step_matches(got, oracle_step(x, 1.0, 0.7), x.cand_offsets, x.block_offsets)
+    assert ctx.device_status() == 0
+    with pytest.raises(binding.SpecsError) as e:
+        ctx.probe_wait_expiry(0)
+    assert e.value.status == 2
