@@ -736,3 +736,50 @@ def test_a_wait_that_nothing_completes_expires_and_is_reported(ctx):
     with pytest.raises(binding.SpecsError) as e:
         ctx.probe_wait_expiry(0)
     assert e.value.status == 2
+
+
+# ------------------------------------------------------------------------------- nothing is written out of bounds
+
+class _Guarded:
+    """A device buffer with 4 KB of a known byte pattern on both sides."""
+    PAD = 4096
+
+    def __init__(self, nbytes, dtype, dev="cuda:0"):
+        self.nbytes = int(nbytes)
+        aligned = (self.nbytes + 255) // 256 * 256
+        self.raw = torch.full((self.PAD + aligned + self.PAD,), 0xA5, dtype=torch.uint8, device=dev)
+        self.view = self.raw[self.PAD:self.PAD + self.nbytes].view(dtype)
+
+    def intact(self):
+        tail = self.raw[self.PAD + self.nbytes:]
+        return bool((self.raw[:self.PAD] == 0xA5).all()) and bool((tail == 0xA5).all())
+
+
+@pytest.mark.parametrize("engine", TC_ENGINES)
+@pytest.mark.parametrize("blk,P,n,d,V", [((1, 1), 1, 1, 8, 8), ((3, 40), 3, 5, 256, 2500), ((129, 129), 1, 1, 64, 1032),
+                                         ((250, 250), 4, 10, 128, 2600)])
+def test_outputs_and_workspace_stay_inside_their_buffers(ctx, engine, blk, P, n, d, V):
+    cfg = small_config("guard", blk, P, n, d, V, seed=6000 + d + V)
+    x = I.make_step_inputs(cfg)
+    s = DeviceStep(ctx, x)
+    rows, B = x.rows, x.blocks
+    g = {"tok": _Guarded(rows * 4, torch.float32), "blk": _Guarded(B * 8, torch.float64),
+         "gen": _Guarded(B * 8, torch.float64), "wts": _Guarded(B * 4, torch.float32),
+         "cho": _Guarded(P * 4, torch.int32), "acc": _Guarded(P, torch.uint8),
+         "ws": _Guarded(ctx.score_workspace_bytes(rows, d, V), torch.uint8),
+         "ids": _Guarded(P * 130 * 4, torch.int32), "len": _Guarded(P * 4, torch.int32)}
+    ctx.set_engine(engine)
+    try:
+        ctx.specs_beam_step(s.hidden, s.w_vocab, s.token_ids, s.block_offsets, s.cand_offsets, s.draft, s.reward,
+                            s.uniforms, 1.0, 0.5, g["tok"].view, g["blk"].view, g["gen"].view, g["wts"].view,
+                            g["cho"].view, g["acc"].view, g["ws"].view)
+        ctx.specs_gather_chosen(s.token_ids, s.block_offsets, s.cand_offsets, g["cho"].view,
+                                g["ids"].view.view(P, 130), g["len"].view)
+        torch.cuda.synchronize()
+    finally:
+        ctx.set_engine(binding.ENGINE_TCGEN05)
+    for name, buf in g.items():
+        assert buf.intact(), f"bytes around `{name}` were overwritten"
+    want = oracle_step(x, 1.0, 0.5)
+    assert np.abs(g["tok"].view.cpu().numpy() - want["tok_logprob"]).max() <= TOK_ATOL
+    assert ctx.device_status() == 0
