@@ -324,6 +324,29 @@ int specs_score_partials(specs_ctx* ctx, const void* hidden, const void* W_shard
 int specs_merge_partials(specs_ctx* ctx, const float* partials, int32_t shards, int64_t rows,
                          const int32_t* token_ids, int32_t V, float* tok_logprob, void* cuda_stream);
 
+/* An 8-bit variant of block scoring (no counterpart in the paper, which states no
+ * precision; an extension for when the LM head is served in FP8).  What it computes:
+ *   1. specs_quantize_rows_e4m3: every row of a bf16 matrix [n, d] is scaled so that its
+ *      largest magnitude maps to 448, the largest finite E4M3 value (OCP 8-bit floating
+ *      point: 1-4-3 bits, bias 7, no infinities), and rounded to the nearest E4M3 number,
+ *      ties to even, saturating: codes uint8 [n, d], scale[n] = absmax / 448 (float32;
+ *      a row of zeros: scale 1, codes 0).  d % 16 == 0.  Weights are quantised once.
+ *   2. specs_score_blocks_fp8: logit[t, v] = hidden_scale[t] * W_scale[v] *
+ *      sum_k hidden_q[t, k] * W_q[v, k] on the tensor cores (tcgen05.mma kind::f8f6f4, fp32
+ *      accumulation, twice the bf16 rate), then the same fused log-softmax, gather, merge
+ *      and block sums as specs_score_blocks; arguments otherwise as there.
+ * Against its own definition (the quantised logits summed exactly) the result meets the
+ * tolerances of the bf16 path; against unquantised bf16 scoring the difference is the
+ * quantisation error, a few percent of the logits' spread. */
+int specs_quantize_rows_e4m3(specs_ctx* ctx, const void* x_bf16, int64_t n, int32_t d,
+                             uint8_t* codes, float* scale, void* cuda_stream);
+size_t specs_score_workspace_bytes_fp8(const specs_ctx* ctx, int64_t rows, int32_t d, int32_t V);
+int specs_score_blocks_fp8(specs_ctx* ctx, const uint8_t* hidden_q, const float* hidden_scale,
+                           const uint8_t* W_q, const float* W_scale, const int32_t* token_ids,
+                           const int64_t* block_offsets, int64_t rows, int32_t d, int32_t V, int32_t B,
+                           float* tok_logprob, float* blk_logprob, double* blk_logprob_f64,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Host-side controller of the SPECS loop (Algorithm 1): for P problems it keeps which
  * model drafts the next n candidate blocks, appends the selected block, applies the
  * dynamic switch (Step III; Section 2.3) and stops at the target length.  All

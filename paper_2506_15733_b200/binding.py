@@ -48,6 +48,10 @@ SIGNATURES = {
                                      C.c_size_t, _vp]),
     "specs_score_partials": (C.c_int, [_vp, _vp, _vp, _vp, _i32, _i64, _i32, _i32, _vp, _vp, C.c_size_t, _vp]),
     "specs_merge_partials": (C.c_int, [_vp, _vp, _i32, _i64, _vp, _i32, _vp, _vp]),
+    "specs_quantize_rows_e4m3": (C.c_int, [_vp, _vp, _i64, _i32, _vp, _vp, _vp]),
+    "specs_score_workspace_bytes_fp8": (C.c_size_t, [_vp, _i64, _i32, _i32]),
+    "specs_score_blocks_fp8": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp,
+                                         C.c_size_t, _vp]),
     "specs_block_sums": (C.c_int, [_vp, _vp, _vp, _i32, _vp, _vp, _vp]),
     "specs_subsample": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _f32, _vp, _vp, _vp, _f32, _vp, _vp]),
     "specs_subsample_f64": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _f32, _vp, _vp, _vp, _f32, _vp, _vp]),
@@ -251,6 +255,26 @@ class Context:
         shards, rows = partials.shape[0], partials.shape[1]
         _check(self._lib.specs_merge_partials(self._h, _ptr(partials), shards, rows, _ptr(token_ids), int(V),
                                               _ptr(tok_logprob), _stream()), "specs_merge_partials")
+
+    def specs_quantize_rows_e4m3(self, x_bf16, codes, scale):
+        """Row-scaled E4M3 quantisation of a bf16 matrix [n, d]: codes uint8 [n, d], scale float32 [n]."""
+        n, d = x_bf16.shape
+        _check(self._lib.specs_quantize_rows_e4m3(self._h, _ptr(x_bf16), n, d, _ptr(codes), _ptr(scale), _stream()),
+               "specs_quantize_rows_e4m3")
+
+    def score_workspace_bytes_fp8(self, rows: int, d: int, V: int) -> int:
+        return int(self._lib.specs_score_workspace_bytes_fp8(self._h, rows, d, V))
+
+    def specs_score_blocks_fp8(self, hidden_q, hidden_scale, w_q, w_scale, token_ids, block_offsets, tok_logprob,
+                               blk_logprob=None, blk_logprob_f64=None, workspace=None):
+        rows, d = hidden_q.shape
+        V = w_q.shape[0]
+        B = block_offsets.shape[0] - 1
+        _check(self._lib.specs_score_blocks_fp8(
+            self._h, _ptr(hidden_q), _ptr(hidden_scale), _ptr(w_q), _ptr(w_scale), _ptr(token_ids),
+            _ptr(block_offsets), rows, d, V, B, _ptr(tok_logprob), _ptr(blk_logprob), _ptr(blk_logprob_f64),
+            _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(), _stream()),
+            "specs_score_blocks_fp8")
 
     def specs_prm_rewards(self, prm_hidden, block_offsets, w_head, bias, reward):
         """Value head of the PRM on each block's last hidden state, logistic link; reward float32 [B] out."""

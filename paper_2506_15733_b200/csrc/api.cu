@@ -25,10 +25,10 @@ double fill_plan(ScorePlan* p, int32_t cta_group, int32_t units) {
     p->units = units;
     p->grid = units * cta_group;
     p->super_tiles = (p->row_tiles + cta_group - 1) / cta_group;
-    const double tile_bytes = (double)kBlockM * cta_group * p->d * 2.0;
+    const double tile_bytes = (double)kBlockM * cta_group * p->d * p->elem_bytes;
     const double t_tile = (double)p->k_blocks * 512.0 / (cta_group == 2 ? kPlanTensorEff2 : kPlanTensorEff1) /
                           kPlanClockHz;
-    const double w_bytes = (double)p->V * p->d * 2.0;
+    const double w_bytes = (double)p->V * p->d * p->elem_bytes;
     auto wave_time = [&](int gm, int s) {
         const int run = (p->vocab_tiles + s - 1) / s;          // vocabulary tiles of the busiest unit
         const double t_hbm = (w_bytes + gm * tile_bytes) / kPlanHbmBytesPerS;
@@ -62,13 +62,15 @@ double fill_plan(ScorePlan* p, int32_t cta_group, int32_t units) {
 }  // namespace
 
 ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t pair_units,
-                          int32_t cta_group, int32_t chunk_kblocks, bool adaptive) {
+                          int32_t cta_group, int32_t chunk_kblocks, bool adaptive, int32_t elem_bytes) {
     ScorePlan p;
     std::memset(&p, 0, sizeof(p));
     p.rows = rows; p.d = d; p.V = V;
     p.row_tiles = (int32_t)((rows + kBlockM - 1) / kBlockM);
     p.vocab_tiles = (V + kBlockN - 1) / kBlockN;
-    p.k_blocks = (d + kBlockK - 1) / kBlockK;
+    p.elem_bytes = elem_bytes;
+    const int32_t k_elems = kBlockK * 2 / elem_bytes;        // elements in a 128-byte k-block
+    p.k_blocks = (d + k_elems - 1) / k_elems;
     p.chunk_kblocks = (chunk_kblocks > 0 && chunk_kblocks < p.k_blocks) ? chunk_kblocks : p.k_blocks;
     p.adaptive = (adaptive && p.chunk_kblocks < p.k_blocks) ? 1 : 0;
     if (pair_units <= 0 && cta_group == 2) cta_group = 1;      // pairs unavailable on this device
@@ -340,6 +342,63 @@ int specs_merge_partials(specs_ctx* ctx, const float* partials, int32_t shards, 
     if (!guard.ok) return SPECS_ERR_CUDA;
     return launch_merge_partials(ctx, partials, shards, rows, token_ids, V, tok_logprob,
                                  static_cast<cudaStream_t>(cuda_stream));
+}
+
+int specs_quantize_rows_e4m3(specs_ctx* ctx, const void* x_bf16, int64_t n, int32_t d, uint8_t* codes, float* scale,
+                             void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    if (n < 0 || d <= 0 || (d % 16) != 0) return SPECS_ERR_SHAPE;
+    if (n == 0) return SPECS_OK;
+    if (!x_bf16 || !codes || !scale) return SPECS_ERR_NULL;
+    if (!aligned16(x_bf16) || !aligned16(codes)) return SPECS_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+    return launch_quantize_rows(x_bf16, n, d, codes, scale, static_cast<cudaStream_t>(cuda_stream));
+}
+
+static ScorePlan fp8_plan(const specs_ctx* ctx, int64_t rows, int32_t d, int32_t V) {
+    const int cta_group = ctx->engine == SPECS_ENGINE_TCGEN05_1CTA ? 1
+                        : ctx->engine == SPECS_ENGINE_TCGEN05_2CTA ? 2 : kCtaGroupAuto;
+    return make_score_plan(rows, d, V, ctx->num_sms, ctx->pair_units, cta_group, ctx->chunk_kblocks,
+                           ctx->accum_adaptive, 1);
+}
+
+size_t specs_score_workspace_bytes_fp8(const specs_ctx* ctx, int64_t rows, int32_t d, int32_t V) {
+    if (!ctx || check_score_shapes(rows, d, V, 0) != SPECS_OK || (d % 16) != 0) return 0;
+    const size_t one = plan_workspace_bytes(make_score_plan(rows, d, V, ctx->num_sms, ctx->pair_units, 1,
+                                                            kDefaultChunkKBlocks, true, 1));
+    const size_t two = plan_workspace_bytes(make_score_plan(rows, d, V, ctx->num_sms, ctx->pair_units, 2,
+                                                            kDefaultChunkKBlocks, true, 1));
+    return one > two ? one : two;
+}
+
+int specs_score_blocks_fp8(specs_ctx* ctx, const uint8_t* hidden_q, const float* hidden_scale, const uint8_t* W_q,
+                           const float* W_scale, const int32_t* token_ids, const int64_t* block_offsets, int64_t rows,
+                           int32_t d, int32_t V, int32_t B, float* tok_logprob, float* blk_logprob,
+                           double* blk_logprob_f64, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    int st = check_score_shapes(rows, d, V, B);
+    if (st != SPECS_OK) return st;
+    if ((d % 16) != 0) return SPECS_ERR_SHAPE;               // rows of 8-bit codes must start on 16-byte boundaries
+    if (!W_q || !W_scale || (B > 0 && !block_offsets)) return SPECS_ERR_NULL;
+    if (rows > 0 && (!hidden_q || !hidden_scale || !token_ids || !tok_logprob || !workspace)) return SPECS_ERR_NULL;
+    if (!aligned16(hidden_q) || !aligned16(W_q) || !aligned16(workspace)) return SPECS_ERR_ALIGN;
+    if (ctx->engine == SPECS_ENGINE_SIMT) return SPECS_ERR_SHAPE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+    if (rows > 0) {
+        const ScorePlan plan = fp8_plan(ctx, rows, d, V);
+        if (workspace_bytes < plan_workspace_bytes(plan)) return SPECS_ERR_WORKSPACE;
+        st = launch_score_tcgen05(ctx, plan, hidden_q, W_q, token_ids, static_cast<float*>(workspace), stream, 0,
+                                  hidden_scale, W_scale);
+        if (st != SPECS_OK) return st;
+        st = launch_merge(ctx, plan, static_cast<const float*>(workspace), token_ids, tok_logprob, stream);
+        if (st != SPECS_OK) return st;
+    }
+    if (B > 0 && (blk_logprob || blk_logprob_f64))
+        return launch_block_sums(tok_logprob, block_offsets, B, blk_logprob, blk_logprob_f64, stream);
+    return SPECS_OK;
 }
 
 int specs_block_sums(specs_ctx* ctx, const float* per_token, const int64_t* block_offsets, int32_t B, float* out,

@@ -233,6 +233,29 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// The same two instructions for 8-bit operands (kind::f8f6f4, K = 32 per instruction).
+__device__ __forceinline__ void tc_mma_f8_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n"
+        "}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_mma_f8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n"
+        "}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                             uint32_t accumulate) {
     asm volatile(
@@ -284,6 +307,10 @@ __device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t saddr) {
     desc |= static_cast<uint64_t>(1) << 46;                   // bits 46-47 descriptor version (sm_100)
     desc |= static_cast<uint64_t>(2) << 61;                   // bits 61-63 swizzle mode: 128 bytes
     return desc;
+}
+// Instruction descriptor of kind::f8f6f4: dense, fp32 accumulate, A and B E4M3 (format code 0), K-major.
+__host__ __device__ constexpr uint32_t instr_desc_e4m3(int m, int n) {
+    return (1u << 4) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
 }
 // Instruction descriptor: dense, fp32 accumulate, A and B bf16, both K-major, M x N.
 __host__ __device__ constexpr uint32_t instr_desc_bf16(int m, int n) {
@@ -352,10 +379,15 @@ __device__ __forceinline__ float read_absmax(const SharedLayout* sh) {
     return m;
 }
 
-template <int kCg>
+// kFp8: operands are E4M3 codes (128 elements per 128-byte k-block, K = 32 per MMA) and the epilogue
+// multiplies every accumulator by hidden_scale[row] * w_scale[column] before anything else.
+template <int kCg, bool kFp8>
 __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, const CUtensorMap& map_w,
                                                  const ScorePlan& plan, const int32_t* __restrict__ token_ids,
-                                                 float* __restrict__ workspace, uint32_t* __restrict__ status) {
+                                                 float* __restrict__ workspace, uint32_t* __restrict__ status,
+                                                 const float* __restrict__ hidden_scale,
+                                                 const float* __restrict__ w_scale) {
+    constexpr int kElemsK = kFp8 ? 2 * kBlockK : kBlockK;    // elements in a 128-byte k-block
     using S = Shape<kCg>;
     constexpr int kStages = S::kStages;
     constexpr uint32_t kStageBytes = S::kStageBytes;
@@ -476,13 +508,13 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                         const uint32_t bar = full0 + stage * 8u;
                         if (kCg == 1) {
                             mbar_arrive_expect_tx(bar, kStageBytes);
-                            tma_load_2d(a_dst, &map_hidden, kb * kBlockK, row0, bar);
-                            tma_load_2d(a_dst + kABytes, &map_w, kb * kBlockK, wrow0, bar);
+                            tma_load_2d(a_dst, &map_hidden, kb * kElemsK, row0, bar);
+                            tma_load_2d(a_dst + kABytes, &map_w, kb * kElemsK, wrow0, bar);
                         } else {
                             // the leader expects both CTAs' bytes; the peer's may be counted first
                             if (rank == 0) mbar_arrive_expect_tx(smem_u32(&sh->full[stage]), 2u * kStageBytes);
-                            tma_load_2d_pair(a_dst, &map_hidden, kb * kBlockK, row0, bar);
-                            tma_load_2d_pair(a_dst + kABytes, &map_w, kb * kBlockK, wrow0, bar);
+                            tma_load_2d_pair(a_dst, &map_hidden, kb * kElemsK, row0, bar);
+                            tma_load_2d_pair(a_dst + kABytes, &map_w, kb * kElemsK, wrow0, bar);
                         }
                         ++issued;
                         if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -517,7 +549,8 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (pair: the leader's)
         if (lane == 0 && rank == 0) {
-            constexpr uint32_t idesc = instr_desc_bf16(kBlockM * kCg, kBlockN);
+            constexpr uint32_t idesc = kFp8 ? instr_desc_e4m3(kBlockM * kCg, kBlockN)
+                                            : instr_desc_bf16(kBlockM * kCg, kBlockN);
             uint32_t stage = 0, phase = 0;
             uint32_t chunk_count = 0;                        // accumulator hand-overs so far
             uint32_t mode_runs = 0;                          // completed phases of the "mode" barrier
@@ -558,15 +591,17 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                             const uint64_t b_desc = smem_desc_k_major_sw128(a_addr + kABytes);
 #pragma unroll
                             for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-                                // advancing 16 bf16 (32 bytes) along K inside the swizzled row: +2 in the
-                                // 16-byte units of the descriptor's start-address field
+                                // advancing 32 bytes (16 bf16 or 32 E4M3) along K inside the swizzled row: +2
+                                // in the 16-byte units of the descriptor's start-address field
                                 const uint32_t accumulate = (kb != kb0 || k != 0) ? 1u : 0u;
-                                if (kCg == 1)
-                                    tc_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                                accumulate);
-                                else
-                                    tc_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k),
-                                                     idesc, accumulate);
+                                const uint64_t a_k = a_desc + (uint64_t)(2 * k), b_k = b_desc + (uint64_t)(2 * k);
+                                if (kFp8) {
+                                    if (kCg == 1) tc_mma_f8(d_tmem, a_k, b_k, idesc, accumulate);
+                                    else          tc_mma_f8_pair(d_tmem, a_k, b_k, idesc, accumulate);
+                                } else {
+                                    if (kCg == 1) tc_mma_bf16(d_tmem, a_k, b_k, idesc, accumulate);
+                                    else          tc_mma_bf16_pair(d_tmem, a_k, b_k, idesc, accumulate);
+                                }
                             }
                             // frees the stage (in both CTAs of a pair) once these MMAs retire
                             if (kCg == 1) tc_commit(smem_u32(&sh->empty[stage]));
@@ -603,6 +638,7 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
             const int64_t row = (int64_t)(st * kCg + (int)rank) * kBlockM + row_in_tile;
             // ids are indices into the whole vocabulary; this W holds rows id_offset .. id_offset + V - 1
             const int32_t id = (row < plan.rows) ? token_ids[row] - plan.id_offset : -1;
+            const float row_scale = (kFp8 && row < plan.rows) ? hidden_scale[row] : 0.0f;
             // state in base-2 units: run_max = max(z) * log2(e), run_sum = sum 2^(z*log2e - run_max)
             float run_max = -INFINITY, run_sum = 0.0f, picked = -INFINITY;
             for (int n = nb; n < ne && ok; ++n) {
@@ -655,6 +691,14 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                 }
                 if (!ok) break;
                 const int col_base = n * kBlockN + half * kHalfN;
+                if (kFp8) {
+                    // de-quantise: the sums are over codes; logit = sum * scale of the row * scale of the column
+#pragma unroll
+                    for (int j = 0; j < kHalfN; ++j) {
+                        const int col = col_base + j;
+                        acc[j] *= row_scale * (col < plan.V ? __ldg(w_scale + col) : 0.0f);
+                    }
+                }
                 if (adapt_run && n == nb) {
                     // first tile of the run: publish this warp's largest |logit| to every CTA of the unit
                     float amax = 0.0f;
@@ -739,14 +783,57 @@ __global__ void __launch_bounds__(kThreads, 1)
 score_tiles_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_w,
                    const ScorePlan plan, const int32_t* __restrict__ token_ids,
                    float* __restrict__ workspace, uint32_t* __restrict__ status) {
-    score_tiles_body<1>(map_hidden, map_w, plan, token_ids, workspace, status);
+    score_tiles_body<1, false>(map_hidden, map_w, plan, token_ids, workspace, status, nullptr, nullptr);
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 score_tiles_pair_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_w,
                         const ScorePlan plan, const int32_t* __restrict__ token_ids,
                         float* __restrict__ workspace, uint32_t* __restrict__ status) {
-    score_tiles_body<2>(map_hidden, map_w, plan, token_ids, workspace, status);
+    score_tiles_body<2, false>(map_hidden, map_w, plan, token_ids, workspace, status, nullptr, nullptr);
+}
+
+// The same two kernels on E4M3 codes with per-row scales.
+__global__ void __launch_bounds__(kThreads, 1)
+score_tiles_fp8_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_w,
+                       const ScorePlan plan, const int32_t* __restrict__ token_ids, float* __restrict__ workspace,
+                       uint32_t* __restrict__ status, const float* __restrict__ hidden_scale,
+                       const float* __restrict__ w_scale) {
+    score_tiles_body<1, true>(map_hidden, map_w, plan, token_ids, workspace, status, hidden_scale, w_scale);
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+score_tiles_pair_fp8_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_w,
+                            const ScorePlan plan, const int32_t* __restrict__ token_ids,
+                            float* __restrict__ workspace, uint32_t* __restrict__ status,
+                            const float* __restrict__ hidden_scale, const float* __restrict__ w_scale) {
+    score_tiles_body<2, true>(map_hidden, map_w, plan, token_ids, workspace, status, hidden_scale, w_scale);
+}
+
+// Row-wise quantisation to E4M3: one warp per row.  scale = absmax / 448; code = nearest E4M3 of
+// x * (448 / absmax), all in float32 with round-to-nearest operations (the codes are integers decided
+// by this arithmetic, so it is spelled out); a row of zeros gets scale 1 and codes 0.
+__global__ void quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t n, int32_t d,
+                                     uint8_t* __restrict__ codes, float* __restrict__ scale) {
+    const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (row >= n) return;
+    const __nv_bfloat16* xr = x + (size_t)row * d;
+    float amax = 0.0f;
+    for (int k = lane; k < d; k += 32) amax = fmaxf(amax, fabsf(__bfloat162float(xr[k])));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    const bool live = amax > 0.0f;
+    const float inv = live ? __fdiv_rn(448.0f, amax) : 1.0f;
+    if (lane == 0) scale[row] = live ? __fdiv_rn(amax, 448.0f) : 1.0f;
+    uint8_t* cr = codes + (size_t)row * d;
+    for (int k = 2 * lane; k < d; k += 64) {                 // d is even: two codes per conversion
+        const float y0 = __fmul_rn(__bfloat162float(xr[k]), inv), y1 = __fmul_rn(__bfloat162float(xr[k + 1]), inv);
+        uint16_t pair;
+        // the first source operand lands in the upper byte, the second in the lower
+        asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(pair) : "f"(y1), "f"(y0));
+        *reinterpret_cast<uint16_t*>(cr + k) = pair;
+    }
 }
 
 // One CTA waits, with the kernel's own bounded wait, on a barrier that nothing ever completes:
@@ -770,13 +857,14 @@ __global__ void wait_expiry_probe_kernel(unsigned long long limit_ns, uint32_t* 
     if (threadIdx.x == 0 && (!completed || abort_flag != 0u)) atomicOr(status, SPECS_DEV_TIMEOUT);
 }
 
-int encode_bf16_2d(specs_ctx* ctx, CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer,
-                   uint32_t box_inner, uint32_t box_outer) {
+int encode_rows_2d(specs_ctx* ctx, CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer,
+                   uint32_t box_inner, uint32_t box_outer, int elem_bytes) {
     const cuuint64_t dims[2] = {inner, outer};
-    const cuuint64_t strides[1] = {inner * 2};               // bytes between consecutive rows
+    const cuuint64_t strides[1] = {inner * (uint64_t)elem_bytes};   // bytes between consecutive rows
     const cuuint32_t box[2] = {box_inner, box_outer};
     const cuuint32_t elem_strides[2] = {1, 1};
-    const CUresult r = ctx->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+    const CUresult r = ctx->encode_tiled(map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                                              : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims,
                                          strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -784,6 +872,14 @@ int encode_bf16_2d(specs_ctx* ctx, CUtensorMap* map, const void* base, uint64_t 
 }
 
 }  // namespace
+
+int launch_quantize_rows(const void* x_bf16, int64_t n, int32_t d, uint8_t* codes, float* scale, cudaStream_t stream) {
+    if (n == 0) return SPECS_OK;
+    const int threads = 256;                                 // eight rows per block
+    quantize_rows_kernel<<<(unsigned)((n + 7) / 8), threads, 0, stream>>>(static_cast<const __nv_bfloat16*>(x_bf16), n,
+                                                                        d, codes, scale);
+    return cuda_status(cudaGetLastError());
+}
 
 int launch_wait_expiry_probe(specs_ctx* ctx, unsigned long long limit_ns, cudaStream_t stream) {
     wait_expiry_probe_kernel<<<1, 64, 0, stream>>>(limit_ns, ctx->d_status);
@@ -803,7 +899,11 @@ int query_pair_units(int device, int num_sms) {
     const bool ok1 = cudaFuncSetAttribute(score_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)Shape<1>::kSmemBytes) == cudaSuccess;
     const bool ok2 = cudaFuncSetAttribute(score_tiles_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)Shape<2>::kSmemBytes) == cudaSuccess &&
+                     cudaFuncSetAttribute(score_tiles_pair_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)Shape<2>::kSmemBytes) == cudaSuccess;
+    cudaFuncSetAttribute(score_tiles_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)Shape<1>::kSmemBytes);
     if (ok2) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(num_sms & ~1), 1, 1);
@@ -826,7 +926,8 @@ int query_pair_units(int device, int num_sms) {
 }
 
 int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan_in, const void* hidden, const void* w_vocab,
-                         const int32_t* token_ids, float* workspace, cudaStream_t stream, int32_t id_offset) {
+                         const int32_t* token_ids, float* workspace, cudaStream_t stream, int32_t id_offset,
+                         const float* hidden_scale, const float* w_scale) {
     static_assert(Shape<1>::kSmemBytes <= 227 * 1024 && Shape<2>::kSmemBytes <= 227 * 1024, "shared memory budget");
     static_assert(Shape<1>::kStages <= kMaxStages && Shape<2>::kStages <= kMaxStages, "barrier arrays");
     static_assert(sizeof(SharedLayout) <= 512, "barrier block");
@@ -839,10 +940,14 @@ int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan_in, const void* h
     plan.id_offset = id_offset;
     query_pair_units(ctx->device, ctx->num_sms);             // shared-memory opt-in for this device
     CUtensorMap map_h, map_w;
-    int st = encode_bf16_2d(ctx, &map_h, hidden, (uint64_t)plan.d, (uint64_t)plan.rows, kBlockK, kBlockM);
+    const bool fp8 = plan.elem_bytes == 1;
+    if (fp8 && (!hidden_scale || !w_scale)) return SPECS_ERR_NULL;
+    const uint32_t box_k = (uint32_t)(kBlockK * 2 / plan.elem_bytes);       // 128 bytes of K
+    int st = encode_rows_2d(ctx, &map_h, hidden, (uint64_t)plan.d, (uint64_t)plan.rows, box_k, kBlockM,
+                            plan.elem_bytes);
     if (st != SPECS_OK) return st;
-    st = encode_bf16_2d(ctx, &map_w, w_vocab, (uint64_t)plan.d, (uint64_t)plan.V, kBlockK,
-                        pair ? Shape<2>::kBRows : Shape<1>::kBRows);
+    st = encode_rows_2d(ctx, &map_w, w_vocab, (uint64_t)plan.d, (uint64_t)plan.V, box_k,
+                        pair ? Shape<2>::kBRows : Shape<1>::kBRows, plan.elem_bytes);
     if (st != SPECS_OK) return st;
 
     TimedLaunch* tl = nullptr;
@@ -856,7 +961,13 @@ int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan_in, const void* h
         tl = &ctx->timed[ctx->timed_used++];
         cudaEventRecord(tl->start, stream);
     }
-    if (pair)
+    if (fp8 && pair)
+        score_tiles_pair_fp8_kernel<<<plan.grid, kThreads, Shape<2>::kSmemBytes, stream>>>(
+            map_h, map_w, plan, token_ids, workspace, ctx->d_status, hidden_scale, w_scale);
+    else if (fp8)
+        score_tiles_fp8_kernel<<<plan.grid, kThreads, Shape<1>::kSmemBytes, stream>>>(
+            map_h, map_w, plan, token_ids, workspace, ctx->d_status, hidden_scale, w_scale);
+    else if (pair)
         score_tiles_pair_kernel<<<plan.grid, kThreads, Shape<2>::kSmemBytes, stream>>>(map_h, map_w, plan, token_ids,
                                                                                       workspace, ctx->d_status);
     else

@@ -39,7 +39,8 @@ struct ScorePlan {
     int32_t d, V;
     int32_t row_tiles;     // ceil(rows / 128)
     int32_t vocab_tiles;   // ceil(V / 256)
-    int32_t k_blocks;      // ceil(d / 64)
+    int32_t k_blocks;      // ceil(d / elements per k-block): 128-byte k-blocks, 64 bf16 or 128 E4M3 elements
+    int32_t elem_bytes;    // 2: bf16 operands; 1: E4M3 operands with per-row scales
     int32_t cta_group;     // CTAs per work unit: 1, or 2 (cluster pair)
     int32_t units;         // work units per wave
     int32_t grid;          // CTAs launched = units * cta_group (also workspace slots per wave)
@@ -66,7 +67,7 @@ constexpr int kCtaGroupAuto = 0;
 // pairs the device can keep resident (<= num_sms / 2; 0: pairs unavailable).
 ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, int32_t pair_units,
                           int32_t cta_group = kCtaGroupAuto, int32_t chunk_kblocks = kDefaultChunkKBlocks,
-                          bool adaptive = true);
+                          bool adaptive = true, int32_t elem_bytes = 2);
 size_t plan_workspace_bytes(const ScorePlan& p);
 // The workspace: triple slots [waves x grid], then one 64-bit progress word per unit.
 __host__ __device__ inline size_t plan_slot_bytes(const ScorePlan& p) {
@@ -124,7 +125,9 @@ namespace specs {
 // device; also opts both kernels in to their dynamic shared memory).  0 if pairs cannot launch.
 int query_pair_units(int device, int num_sms);
 int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan, const void* hidden, const void* w_vocab,
-                         const int32_t* token_ids, float* workspace, cudaStream_t stream, int32_t id_offset = 0);
+                         const int32_t* token_ids, float* workspace, cudaStream_t stream, int32_t id_offset = 0,
+                         const float* hidden_scale = nullptr, const float* w_scale = nullptr);
+int launch_quantize_rows(const void* x_bf16, int64_t n, int32_t d, uint8_t* codes, float* scale, cudaStream_t stream);
 int launch_wait_expiry_probe(specs_ctx* ctx, unsigned long long limit_ns, cudaStream_t stream);
 int launch_score_simt(specs_ctx* ctx, const void* hidden, const void* w_vocab, const int32_t* token_ids,
                       int64_t rows, int32_t d, int32_t V, float* tok_logprob, cudaStream_t stream);

@@ -1,0 +1,92 @@
+"""GPU parity of the E4M3 variant: the quantiser bit for bit, the scoring within the bf16 path's
+tolerances against the quantised definition computed exactly by the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import specs_fp8 as F
+from oracle import specs_oracle as O
+from paper_2506_15733_b200 import binding
+from paper_2506_15733_b200 import inputs as I
+from tests.gpu_util import BLK_RTOL, TOK_ATOL
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(0)
+    yield c
+    assert c.device_status() == 0
+    c.close()
+
+
+def quantize_on_gpu(ctx, bits):
+    x = binding.bf16_bits_to_device(bits, DEV)
+    codes = torch.full(x.shape, 0x55, dtype=torch.uint8, device=DEV)
+    scale = torch.full((x.shape[0],), -1.0, dtype=torch.float32, device=DEV)
+    ctx.specs_quantize_rows_e4m3(x, codes, scale)
+    return codes, scale
+
+
+@pytest.mark.parametrize("n,d,scale", [(37, 16, 1.0), (300, 272, 5.0), (64, 3584, 0.02)])
+def test_quantiser_is_bit_exact(ctx, n, d, scale):
+    cfg = I.StepConfig("q", 7400 + d, 1, 1, (n, n), d, 16, 0.05, hidden_scale=scale)
+    x = I.make_step_inputs(cfg)
+    bits = x.hidden.copy()
+    bits[3] = 0                                                   # a row of zeros
+    bits[5, 1:] = 0                                               # a single non-zero element
+    codes, sc = quantize_on_gpu(ctx, bits)
+    torch.cuda.synchronize()
+    want_c, want_s = F.quantize_rows(bits)
+    assert np.array_equal(codes.cpu().numpy(), want_c)
+    assert np.array_equal(sc.cpu().numpy(), want_s)
+
+
+@pytest.mark.parametrize("engine", [binding.ENGINE_TCGEN05_1CTA, binding.ENGINE_TCGEN05_2CTA])
+@pytest.mark.parametrize("blk,P,n,d,V", [((1, 1), 1, 1, 16, 8), ((3, 40), 3, 5, 272, 2500), ((129, 129), 1, 1, 128, 1032),
+                                         ((250, 250), 4, 10, 256, 2600)])
+def test_fp8_scoring_matches_its_definition(ctx, engine, blk, P, n, d, V):
+    cfg = I.StepConfig("f8", 7500 + d + V, P, n, blk, d, V, 0.05)
+    x = I.make_step_inputs(cfg)
+    hq, hs = quantize_on_gpu(ctx, x.hidden)
+    wq, ws_ = quantize_on_gpu(ctx, x.w_vocab)
+    tok = torch.full((x.rows,), float("nan"), dtype=torch.float32, device=DEV)
+    blk64 = torch.full((x.blocks,), float("nan"), dtype=torch.float64, device=DEV)
+    work = torch.empty(max(ctx.score_workspace_bytes_fp8(x.rows, d, V), 16), dtype=torch.uint8, device=DEV)
+    ctx.set_engine(engine)
+    try:
+        ctx.specs_score_blocks_fp8(hq, hs, wq, ws_, torch.from_numpy(x.token_ids).to(DEV),
+                                   torch.from_numpy(x.block_offsets).to(DEV), tok, None, blk64, work)
+        torch.cuda.synchronize()
+    finally:
+        ctx.set_engine(binding.ENGINE_TCGEN05)
+    qh, sh = F.quantize_rows(x.hidden)
+    qw, sw = F.quantize_rows(x.w_vocab)
+    want = F.token_logprobs_fp8(qh, sh, qw, sw, x.token_ids)
+    got = tok.cpu().numpy()
+    assert np.abs(got - want).max() <= TOK_ATOL
+    want_blk = O.block_sums(want, x.block_offsets)
+    nz = want_blk != 0
+    assert np.all(np.abs(blk64.cpu().numpy()[nz] - want_blk[nz]) <= BLK_RTOL * np.abs(want_blk[nz]))
+    # and it is the quantisation, not the kernel, that separates it from the bf16 result
+    exact = O.token_logprobs(x.hidden, x.w_vocab, x.token_ids)
+    assert np.abs(got - exact).max() < 0.3
+    assert ctx.device_status() == 0
+
+
+def test_fp8_argument_checks(ctx):
+    h = torch.zeros((4, 24), dtype=torch.uint8, device=DEV)       # d % 16 != 0
+    s = torch.ones(4, dtype=torch.float32, device=DEV)
+    ids = torch.zeros(4, dtype=torch.int32, device=DEV)
+    off = torch.tensor([0, 4], dtype=torch.int64, device=DEV)
+    tok = torch.zeros(4, dtype=torch.float32, device=DEV)
+    ws = torch.empty(1 << 20, dtype=torch.uint8, device=DEV)
+    with pytest.raises(binding.SpecsError) as e:
+        ctx.specs_score_blocks_fp8(h, s, h, s, ids, off, tok, None, None, ws)
+    assert e.value.status == 2
+    h = torch.zeros((4, 32), dtype=torch.uint8, device=DEV)
+    with pytest.raises(binding.SpecsError) as e:
+        ctx.specs_score_blocks_fp8(h, None, h, s, ids, off, tok, None, None, ws)
+    assert e.value.status == 1
