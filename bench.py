@@ -176,6 +176,9 @@ def main():
                     help="pacing of the CTA pairs that stream the same W chunk, in vocabulary tiles (0: off; default: the library's)")
     ap.add_argument("--time-every", type=int, default=1,
                     help="record CUDA events around the scoring kernel on every K-th step of the timed region")
+    ap.add_argument("--fp8", action="store_true",
+                    help="time the E4M3 variant instead (reduced precision: not the headline; W quantised once, "
+                         "hidden states quantised inside every step)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -230,6 +233,22 @@ def main():
     def step():
         ctx.specs_beam_step(hidden, w_vocab, ids, boff, coff, draft, reward, uni, beta, tau, tok, blk64, gen64, wts,
                             chosen, accept, ws)
+
+    if args.fp8:
+        w_q = torch.empty((V, d), dtype=torch.uint8, device=dev)
+        w_s = torch.empty(V, dtype=torch.float32, device=dev)
+        ctx.specs_quantize_rows_e4m3(w_vocab, w_q, w_s)          # the weight is quantised once, outside the step
+        h_q = torch.empty((rows, d), dtype=torch.uint8, device=dev)
+        h_s = torch.empty(rows, dtype=torch.float32, device=dev)
+        ws = torch.empty(ctx.score_workspace_bytes_fp8(rows, d, V), dtype=torch.uint8, device=dev)
+        launches_per_step = 6   # quantise hidden; score tiles; merge; target block sums; generator block sums; SubSample
+        args.no_e2e = True
+
+        def step():  # noqa: F811
+            ctx.specs_quantize_rows_e4m3(hidden, h_q, h_s)
+            ctx.specs_score_blocks_fp8(h_q, h_s, w_q, w_s, ids, boff, tok, None, blk64, ws)
+            ctx.specs_block_sums(draft, boff, None, gen64)
+            ctx.specs_subsample(blk64, gen64, reward, coff, beta, uni, chosen, wts, tau, accept)
 
     def barrier():
         ranks.barrier()
@@ -313,16 +332,23 @@ def main():
         peaks = load_peaks()
         flops = 2.0 * rows * d * V
         achieved = flops / (kernel_ms * 1e-3) / 1e12 if kernel_ms > 0 else None
-        peak = peaks["bf16_tflops_sustained"]
         plan = binding.score_plan(rows, d, V, ctx.sm_count())
+        nominal = NOMINAL_BF16_TFLOPS
+        if args.fp8:                                             # E4M3 runs at twice the bf16 rate
+            peaks = {k: (2.0 * v if k.startswith("bf16") else v) for k, v in peaks.items()}
+            peaks["source"] = "measured bf16 x 2 (nominal fp8 : bf16 ratio)" if peaks["source"] == "measured" else "fallback x 2"
+            nominal = 2.0 * NOMINAL_BF16_TFLOPS
+        peak = peaks["bf16_tflops_sustained"]
         roofline = {"bound": "tensor",
-                    "kernel": "score_tiles_pair_kernel" if plan["cta_group"] == 2 else "score_tiles_kernel", "achieved": achieved, "peak": peak,
+                    "kernel": ("score_tiles_pair" if plan["cta_group"] == 2 else "score_tiles") +
+                              ("_fp8_kernel" if args.fp8 else "_kernel"), "achieved": achieved, "peak": peak,
                     "unit": "TFLOP/s", "frac": achieved / peak if achieved else None,
-                    "peak_kind": f"bf16 sustained, of {peaks['source']} (kernel timed inside a long loop)",
+                    "peak_kind": f"{'fp8' if args.fp8 else 'bf16'} sustained, of {peaks['source']} "
+                                 "(kernel timed inside a long loop)",
                     "frac_of_burst": achieved / peaks["bf16_tflops"] if achieved else None,
-                    "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS if achieved else None,
+                    "frac_of_nominal": achieved / nominal if achieved else None,
                     "kernel_ms": kernel_ms, "kernel_launches_timed": kernel_launches,
-                    "flop_per_launch": flops, "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
+                    "flop_per_launch": flops, "traffic": None if args.fp8 else NCU_TRAFFIC_BYTES.get(cfg.name),
                     "burst": {"steps": burst_steps, "ms_per_step": burst_ms, "kernel_ms": burst_kernel_ms,
                               "achieved": flops / (burst_kernel_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"],
                               "frac": flops / (burst_kernel_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
@@ -341,7 +367,7 @@ def main():
                              f"{reps} times: {total_dt:.1f} s of fp64 numpy incl. bf16->fp64 decode of W"}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "scaling": "weak", "vs_baseline": None, "dtype": "e4m3" if args.fp8 else "bf16", "data": "synthetic",
                 "config": {"workload": cfg.name, "rows": rows, "blocks": B, "problems": P, "d": d, "V": V,
                            "beta": beta, "tau": tau, "l2": f"inputs exceed L2 (W_vocab {V * d * 2 / 1e9:.2f} GB vs 126 MB); no flush",
                            "parallelism": f"replicas x{world}, no collective"},

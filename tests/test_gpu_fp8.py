@@ -90,3 +90,33 @@ def test_fp8_argument_checks(ctx):
     with pytest.raises(binding.SpecsError) as e:
         ctx.specs_score_blocks_fp8(h, None, h, s, ids, off, tok, None, None, ws)
     assert e.value.status == 1
+
+
+def test_fp8_scoring_at_the_7b_shape(ctx):
+    cfg = I.CONFIGS["step7b"]
+    x = I.make_step_inputs(cfg)
+    hq, hs = quantize_on_gpu(ctx, x.hidden)
+    wq, ws_ = quantize_on_gpu(ctx, x.w_vocab)
+    tok = torch.full((x.rows,), float("nan"), dtype=torch.float32, device=DEV)
+    work = torch.empty(ctx.score_workspace_bytes_fp8(x.rows, cfg.d, cfg.vocab), dtype=torch.uint8, device=DEV)
+    ids, off = torch.from_numpy(x.token_ids).to(DEV), torch.from_numpy(x.block_offsets).to(DEV)
+    ctx.specs_score_blocks_fp8(hq, hs, wq, ws_, ids, off, tok, None, None, work)
+    torch.cuda.synchronize()
+    got = tok.cpu().numpy()
+    assert np.all(np.isfinite(got))
+    # the GPU's codes are the oracle's (checked bit for bit on W, which is the large one)
+    qw, sw = F.quantize_rows(x.w_vocab)
+    assert np.array_equal(wq.cpu().numpy(), qw) and np.array_equal(ws_.cpu().numpy(), sw)
+    rows = np.arange(0, x.rows, 8)                                # every eighth row through the oracle
+    qh, sh = F.quantize_rows(x.hidden[rows])
+    want = F.token_logprobs_fp8(qh, sh, qw, sw, x.token_ids[rows])
+    assert np.abs(got[rows] - want).max() <= TOK_ATOL
+    # timing, for the record of this test's log
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(50):
+        ctx.specs_score_blocks_fp8(hq, hs, wq, ws_, ids, off, tok, None, None, work)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / 50
+    print(f"fp8 scoring of {x.rows} rows: {ms:.3f} ms per call, {2.0 * x.rows * cfg.d * cfg.vocab / ms / 1e9:.0f} TFLOP/s")
