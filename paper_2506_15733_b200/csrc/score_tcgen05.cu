@@ -49,6 +49,18 @@
 // tile on the MMA issuer and the epilogue both derive the chunk length from it
 // (adaptive_chunk_kblocks).  The hand-over is a barrier ("mode") on which every epilogue warp of
 // the unit arrives after writing its maximum into every CTA of the unit.
+//
+// Pacing: the units (CTAs or pairs) that own the same vocabulary chunk in a wave read the same W
+// tiles.  Only while they stay within about a tile of each other does a tile come from HBM once and
+// from L2 for the others; left alone they drift apart within milliseconds and every tile is fetched
+// several times.  Each unit therefore publishes its progress in a 64-bit word behind the workspace's
+// slots and does not start tile t before all units of its chunk have started tile t - lead.  The
+// wait is advisory (bounded, gives up for good after a few expiries).
+//
+// 8-bit operands (template parameter kFp8): the same kernel on E4M3 codes with per-row scales,
+// 128 elements per k-block, tcgen05.mma kind::f8f6f4; the epilogue first multiplies each
+// accumulator by scale of the row x scale of the column.
+//
 // Every mbarrier wait is bounded; on expiry the CTA raises SPECS_DEV_TIMEOUT, all roles leave
 // their loops, the producer waits (bounded) for its copies in flight, TMEM is freed and the
 // kernel returns.
