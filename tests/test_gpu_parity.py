@@ -783,3 +783,39 @@ def test_outputs_and_workspace_stay_inside_their_buffers(ctx, engine, blk, P, n,
     want = oracle_step(x, 1.0, 0.5)
     assert np.abs(g["tok"].view.cpu().numpy() - want["tok_logprob"]).max() <= TOK_ATOL
     assert ctx.device_status() == 0
+
+
+# ------------------------------------------------------------------------------- seeded random shapes
+
+def _random_shapes(count, seed):
+    rng = np.random.Generator(np.random.Philox(key=[seed, 9]))
+    out = []
+    for _ in range(count):
+        d = int(rng.integers(1, 80)) * 8                            # any multiple of 8 up to 632 (k-block tails)
+        V = int(rng.integers(1, 3000))
+        P = int(rng.integers(1, 6))
+        n = int(rng.integers(1, 9))
+        hi = int(rng.integers(1, 120))
+        lo = int(rng.integers(0, hi + 1))
+        out.append((d, V, P, n, lo, hi, int(rng.integers(0, 3))))
+    return out
+
+
+@pytest.mark.parametrize("d,V,P,n,lo,hi,mode", _random_shapes(24, 6100))
+def test_random_shapes_against_the_oracle(ctx, d, V, P, n, lo, hi, mode):
+    cfg = small_config("fuzz", (lo, hi), P, n, d, V, seed=6100 + d + V, w_sigma=0.6 / math.sqrt(d) * (1 + mode))
+    x = I.make_step_inputs(cfg)
+    if x.rows == 0:
+        pytest.skip("all blocks empty")
+    engine = [binding.ENGINE_TCGEN05, binding.ENGINE_TCGEN05_1CTA, binding.ENGINE_TCGEN05_2CTA][mode]
+    ctx.set_engine(engine)
+    try:
+        sep = DeviceStep(ctx, x).step(1.3, 0.6)
+        fused = _fused_step(ctx, DeviceStep(ctx, x), 1.3, 0.6)
+    finally:
+        ctx.set_engine(binding.ENGINE_TCGEN05)
+    want = oracle_step(x, 1.3, 0.6)
+    assert_step_matches(sep, want, x.cand_offsets, x.block_offsets)
+    for key in ("tok_logprob", "blk_logprob_f64", "blk_logprob_gen", "weights", "chosen", "accept"):
+        assert np.array_equal(fused[key], sep[key]), key
+    assert ctx.device_status() == 0
