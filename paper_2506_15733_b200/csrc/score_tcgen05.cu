@@ -363,17 +363,21 @@ struct SharedLayout {
     uint32_t abort_flag;
 };
 
-// Chunk length (in k-blocks of 64) for logits whose magnitude stays below twice `absmax`.
-// One accumulation (K = 16) truncates the fp32 accumulator toward zero by at most one spacing of
-// its magnitude.  The chunk gets as many accumulations as keep (count x spacing) under 2.5e-4,
-// an eighth of the 2e-3 tolerance on a token log-probability; it is never shorter than `base`.
-// `*bound` receives the magnitude up to which that spacing holds (the top of the binade).
+// Chunk length (in k-blocks) for logits whose magnitude stays below twice `absmax`.
+// One accumulation (one MMA instruction along K) truncates the fp32 accumulator toward zero by at most
+// one spacing of its magnitude.  The chunk gets as many accumulations as keep (count x spacing at twice
+// the sampled magnitude) under 1e-3, half of the 2e-3 tolerance on a token log-probability.  That product
+// is a worst case: the loss per accumulation averages half a spacing, and of the partial sum's magnitude,
+// not the final one's; measured, the bias is about a quarter of it (-5e-3 at |logit| = 700, d = 5120,
+// one chunk: bound 2e-2), and another factor of two is the margin on the sampled magnitude.  The chunk is
+// never shorter than `base`.  `*bound` receives the magnitude up to which that spacing holds (the top of
+// the binade).
 __device__ __forceinline__ int adaptive_chunk_kblocks(float absmax, int base, int k_blocks, float* bound) {
     *bound = INFINITY;                                       // no claim when the base chunk is kept
     const float a = fmaxf(2.0f * absmax, 1.0f);
-    if (!(a < 128.0f)) return base;                          // also NaN and inf
+    if (!(a < 1024.0f)) return base;                         // also NaN and inf
     const int e = ((__float_as_int(a) >> 23) & 0xff) - 126;  // a = m * 2^e with m in [0.5, 1)
-    const float n_acc = ldexpf(2.5e-4f, 24 - e);             // spacing of [2^(e-1), 2^e) is 2^(e-24)
+    const float n_acc = ldexpf(1.0e-3f, 24 - e);             // spacing of [2^(e-1), 2^e) is 2^(e-24)
     int kb = (int)(n_acc * 0.25f);                           // four accumulations per k-block
     if (kb <= base) return base;
     *bound = ldexpf(1.0f, e);

@@ -389,7 +389,7 @@ def _score_only(ctx, x):
     return s.tok_lp.cpu().numpy()
 
 
-@pytest.mark.parametrize("sigma_z", [1.5, 3.0, 6.0, 12.0])
+@pytest.mark.parametrize("sigma_z", [1.5, 3.0, 6.0, 12.0, 24.0, 48.0])
 def test_adaptive_chunks_keep_the_tolerance_across_logit_magnitudes(ctx, sigma_z):
     # long reduction (d = 5120), runs of at least three vocabulary tiles per work unit, and logit scales
     # that land in different chunk lengths (unchunked ... 1024 elements ... the 512-element base)
