@@ -340,7 +340,9 @@ int specs_merge_partials(specs_ctx* ctx, const float* partials, int32_t shards, 
  *      and block sums as specs_score_blocks; arguments otherwise as there.
  * Against its own definition (the quantised logits summed exactly) the result meets the
  * tolerances of the bf16 path; against unquantised bf16 scoring the difference is the
- * quantisation error, a few percent of the logits' spread. */
+ * quantisation error, a few percent of the logits' spread.  Accumulation chunks are
+ * counted in 128-byte k-blocks, so a length set with specs_set_accum_chunk covers
+ * twice as many elements here (the default base chunk is 1024 elements). */
 int specs_quantize_rows_e4m3(specs_ctx* ctx, const void* x_bf16, int64_t n, int32_t d,
                              uint8_t* codes, float* scale, void* cuda_stream);
 size_t specs_score_workspace_bytes_fp8(const specs_ctx* ctx, int64_t rows, int32_t d, int32_t V);
