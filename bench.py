@@ -238,17 +238,13 @@ def main():
         w_q = torch.empty((V, d), dtype=torch.uint8, device=dev)
         w_s = torch.empty(V, dtype=torch.float32, device=dev)
         ctx.specs_quantize_rows_e4m3(w_vocab, w_q, w_s)          # the weight is quantised once, outside the step
-        h_q = torch.empty((rows, d), dtype=torch.uint8, device=dev)
-        h_s = torch.empty(rows, dtype=torch.float32, device=dev)
-        ws = torch.empty(ctx.score_workspace_bytes_fp8(rows, d, V), dtype=torch.uint8, device=dev)
-        launches_per_step = 6   # quantise hidden; score tiles; merge; target block sums; generator block sums; SubSample
+        ws = torch.empty(ctx.beam_step_fp8_workspace_bytes(rows, d, V), dtype=torch.uint8, device=dev)
+        launches_per_step = 3   # quantise the hidden states; score tiles; finish
         args.no_e2e = True
 
         def step():  # noqa: F811
-            ctx.specs_quantize_rows_e4m3(hidden, h_q, h_s)
-            ctx.specs_score_blocks_fp8(h_q, h_s, w_q, w_s, ids, boff, tok, None, blk64, ws)
-            ctx.specs_block_sums(draft, boff, None, gen64)
-            ctx.specs_subsample(blk64, gen64, reward, coff, beta, uni, chosen, wts, tau, accept)
+            ctx.specs_beam_step_fp8(hidden, w_q, w_s, ids, boff, coff, draft, reward, uni, beta, tau, tok, blk64, gen64,
+                                    wts, chosen, accept, ws)
 
     def barrier():
         ranks.barrier()

@@ -352,6 +352,20 @@ int specs_score_blocks_fp8(specs_ctx* ctx, const uint8_t* hidden_q, const float*
                            float* tok_logprob, float* blk_logprob, double* blk_logprob_f64,
                            void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* The whole beam step with the 8-bit head, in three launches: quantise the step's
+ * hidden states (bf16 [rows, d] in), score them against the pre-quantised weight,
+ * and the finish kernel of specs_beam_step.  Arguments as in specs_beam_step, with
+ * W_q / W_scale from specs_quantize_rows_e4m3; the workspace also holds the codes and
+ * scales of the hidden states (specs_beam_step_fp8_workspace_bytes). */
+size_t specs_beam_step_fp8_workspace_bytes(const specs_ctx* ctx, int64_t rows, int32_t d, int32_t V);
+int specs_beam_step_fp8(specs_ctx* ctx, const void* hidden, const uint8_t* W_q, const float* W_scale,
+                        const int32_t* token_ids, const int64_t* block_offsets, const int32_t* cand_offsets,
+                        const float* gen_tok_logprob, const float* reward, const float* uniforms,
+                        int64_t rows, int32_t d, int32_t V, int32_t B, int32_t P, float beta, float tau,
+                        float* tok_logprob, double* blk_logprob_f64, double* gen_blk_logprob_f64,
+                        float* weights, int32_t* chosen, uint8_t* accept,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Host-side controller of the SPECS loop (Algorithm 1): for P problems it keeps which
  * model drafts the next n candidate blocks, appends the selected block, applies the
  * dynamic switch (Step III; Section 2.3) and stops at the target length.  All

@@ -52,6 +52,9 @@ SIGNATURES = {
     "specs_score_workspace_bytes_fp8": (C.c_size_t, [_vp, _i64, _i32, _i32]),
     "specs_score_blocks_fp8": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp,
                                          C.c_size_t, _vp]),
+    "specs_beam_step_fp8_workspace_bytes": (C.c_size_t, [_vp, _i64, _i32, _i32]),
+    "specs_beam_step_fp8": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32,
+                                      _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_size_t, _vp]),
     "specs_block_sums": (C.c_int, [_vp, _vp, _vp, _i32, _vp, _vp, _vp]),
     "specs_subsample": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _f32, _vp, _vp, _vp, _f32, _vp, _vp]),
     "specs_subsample_f64": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _i32, _f32, _vp, _vp, _vp, _f32, _vp, _vp]),
@@ -275,6 +278,24 @@ class Context:
             _ptr(block_offsets), rows, d, V, B, _ptr(tok_logprob), _ptr(blk_logprob), _ptr(blk_logprob_f64),
             _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(), _stream()),
             "specs_score_blocks_fp8")
+
+    def beam_step_fp8_workspace_bytes(self, rows: int, d: int, V: int) -> int:
+        return int(self._lib.specs_beam_step_fp8_workspace_bytes(self._h, rows, d, V))
+
+    def specs_beam_step_fp8(self, hidden, w_q, w_scale, token_ids, block_offsets, cand_offsets, gen_tok_logprob, reward,
+                            uniforms, beta, tau, tok_logprob, blk_logprob_f64, gen_blk_logprob_f64, weights, chosen,
+                            accept, workspace):
+        """The whole step with the 8-bit head: quantise the hidden states, score, finish."""
+        rows, d = hidden.shape
+        V = w_q.shape[0]
+        B = block_offsets.shape[0] - 1
+        P = cand_offsets.shape[0] - 1
+        _check(self._lib.specs_beam_step_fp8(
+            self._h, _ptr(hidden), _ptr(w_q), _ptr(w_scale), _ptr(token_ids), _ptr(block_offsets), _ptr(cand_offsets),
+            _ptr(gen_tok_logprob), _ptr(reward), _ptr(uniforms), rows, d, V, B, P, float(beta), float(tau),
+            _ptr(tok_logprob), _ptr(blk_logprob_f64), _ptr(gen_blk_logprob_f64), _ptr(weights), _ptr(chosen),
+            _ptr(accept), _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
+            _stream()), "specs_beam_step_fp8")
 
     def specs_prm_rewards(self, prm_hidden, block_offsets, w_head, bias, reward):
         """Value head of the PRM on each block's last hidden state, logistic link; reward float32 [B] out."""

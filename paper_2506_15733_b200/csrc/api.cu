@@ -401,6 +401,61 @@ int specs_score_blocks_fp8(specs_ctx* ctx, const uint8_t* hidden_q, const float*
     return SPECS_OK;
 }
 
+// layout of the fused 8-bit step's workspace: [codes of the hidden states | their scales | scoring workspace]
+static size_t fp8_step_offsets(int64_t rows, int32_t d, size_t* off_scale, size_t* off_ws) {
+    const size_t codes = ((size_t)rows * d + 255) & ~(size_t)255;
+    const size_t scales = ((size_t)rows * sizeof(float) + 255) & ~(size_t)255;
+    *off_scale = codes;
+    *off_ws = codes + scales;
+    return codes + scales;
+}
+
+size_t specs_beam_step_fp8_workspace_bytes(const specs_ctx* ctx, int64_t rows, int32_t d, int32_t V) {
+    const size_t ws = specs_score_workspace_bytes_fp8(ctx, rows, d, V);
+    if (ws == 0) return 0;
+    size_t o1, o2;
+    return fp8_step_offsets(rows, d, &o1, &o2) + ws;
+}
+
+int specs_beam_step_fp8(specs_ctx* ctx, const void* hidden, const uint8_t* W_q, const float* W_scale,
+                        const int32_t* token_ids, const int64_t* block_offsets, const int32_t* cand_offsets,
+                        const float* gen_tok_logprob, const float* reward, const float* uniforms, int64_t rows,
+                        int32_t d, int32_t V, int32_t B, int32_t P, float beta, float tau, float* tok_logprob,
+                        double* blk_logprob_f64, double* gen_blk_logprob_f64, float* weights, int32_t* chosen,
+                        uint8_t* accept, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!ctx) return SPECS_ERR_NULL;
+    int st = check_score_shapes(rows, d, V, B);
+    if (st != SPECS_OK) return st;
+    if (P < 0 || (d % 16) != 0) return SPECS_ERR_SHAPE;
+    if (P == 0) return SPECS_OK;
+    if (!W_q || !W_scale || !block_offsets || !cand_offsets || !chosen) return SPECS_ERR_NULL;
+    if (rows > 0 && (!hidden || !token_ids || !tok_logprob || !workspace)) return SPECS_ERR_NULL;
+    if (B > 0 && (!reward || !uniforms || !blk_logprob_f64 || (gen_tok_logprob && !gen_blk_logprob_f64)))
+        return SPECS_ERR_NULL;
+    if (!aligned16(hidden) || !aligned16(W_q) || !aligned16(workspace)) return SPECS_ERR_ALIGN;
+    if (ctx->engine == SPECS_ENGINE_SIMT) return SPECS_ERR_SHAPE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+
+    const ScorePlan plan = fp8_plan(ctx, rows, d, V);
+    size_t off_scale, off_ws;
+    const size_t head = fp8_step_offsets(rows, d, &off_scale, &off_ws);
+    uint8_t* base = static_cast<uint8_t*>(workspace);
+    float* ws = reinterpret_cast<float*>(base + off_ws);
+    if (rows > 0) {
+        if (workspace_bytes < head + plan_workspace_bytes(plan)) return SPECS_ERR_WORKSPACE;
+        float* h_scale = reinterpret_cast<float*>(base + off_scale);
+        st = launch_quantize_rows(hidden, rows, d, base, h_scale, stream);
+        if (st != SPECS_OK) return st;
+        st = launch_score_tcgen05(ctx, plan, base, W_q, token_ids, ws, stream, 0, h_scale, W_scale);
+        if (st != SPECS_OK) return st;
+    }
+    return launch_finish_step(ctx, plan, ws, nullptr, nullptr, token_ids, block_offsets, cand_offsets, P,
+                              const_cast<float*>(gen_tok_logprob), reward, uniforms, beta, tau, tok_logprob,
+                              blk_logprob_f64, gen_blk_logprob_f64, weights, chosen, accept, nullptr, nullptr, 0, stream);
+}
+
 int specs_block_sums(specs_ctx* ctx, const float* per_token, const int64_t* block_offsets, int32_t B, float* out,
                      double* out_f64, void* cuda_stream) {
     if (!ctx) return SPECS_ERR_NULL;

@@ -120,3 +120,35 @@ def test_fp8_scoring_at_the_7b_shape(ctx):
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / 50
     print(f"fp8 scoring of {x.rows} rows: {ms:.3f} ms per call, {2.0 * x.rows * cfg.d * cfg.vocab / ms / 1e9:.0f} TFLOP/s")
+
+
+def test_fused_fp8_step_equals_the_separate_calls_and_the_oracle(ctx):
+    from tests.gpu_util import DeviceStep, assert_step_matches
+    cfg = I.StepConfig("f8step", 7600, 3, 5, (3, 60), 272, 2500, 0.05)
+    x = I.make_step_inputs(cfg)
+    s = DeviceStep(ctx, x)
+    wq, wsc = quantize_on_gpu(ctx, x.w_vocab)
+    work = torch.empty(ctx.beam_step_fp8_workspace_bytes(x.rows, 272, 2500), dtype=torch.uint8, device=DEV)
+    ctx.specs_beam_step_fp8(s.hidden, wq, wsc, s.token_ids, s.block_offsets, s.cand_offsets, s.draft, s.reward,
+                            s.uniforms, 1.0, 0.6, s.tok_lp, s.blk_lp64, s.gen_blk64, s.weights, s.chosen, s.accept, work)
+    torch.cuda.synchronize()
+    got = s.results()
+    # separate calls on the same codes
+    hq, hs = quantize_on_gpu(ctx, x.hidden)
+    tok = torch.empty(x.rows, dtype=torch.float32, device=DEV)
+    w2 = torch.empty(ctx.score_workspace_bytes_fp8(x.rows, 272, 2500), dtype=torch.uint8, device=DEV)
+    ctx.specs_score_blocks_fp8(hq, hs, wq, wsc, s.token_ids, s.block_offsets, tok, None, None, w2)
+    torch.cuda.synchronize()
+    assert np.array_equal(tok.cpu().numpy(), got["tok_logprob"])
+    # the oracle's step on the quantised definition
+    qh, sh = F.quantize_rows(x.hidden)
+    qw, sw = F.quantize_rows(x.w_vocab)
+    lp = F.token_logprobs_fp8(qh, sh, qw, sw, x.token_ids)
+    LP, LQ = O.block_sums(lp, x.block_offsets), O.block_sums(x.draft_tok_logprob, x.block_offsets)
+    S = O.scores(LP, LQ, x.reward, 1.0)
+    chosen, margin = O.gumbel_pick(S, x.uniforms, x.cand_offsets)
+    want = {"tok_logprob": lp, "blk_logprob": LP, "chosen": chosen, "margin": margin,
+            "accept": O.accept_flags(x.reward, x.cand_offsets, 0.6)}
+    got["blk_logprob"] = got["blk_logprob_f64"].astype(np.float32)
+    assert_step_matches(got, want, x.cand_offsets, x.block_offsets)
+    assert ctx.device_status() == 0
