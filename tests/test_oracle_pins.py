@@ -411,3 +411,23 @@ def test_accept_flag_laws():
     c2 = np.array([0, 2, 2, 4], dtype=np.int32)
     assert O.accept_flags(r2, c2, np.float32(0.7)).tolist() == [0, 0, 1]
     assert O.accept_flags(r2, c2, 0.69).tolist() == [1, 0, 1]
+
+
+def test_oracle_reproduces_its_stored_tiny_step():
+    # regression anchor written by tests/golden/make_tiny_step_golden.py (which calls only the oracle)
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "tiny_step.txt")
+    stored = {}
+    for line in open(path):
+        if line.startswith("#"):
+            continue
+        key, *vals = line.split()
+        stored[key] = vals
+    x = I.make_step_inputs(I.CONFIGS["tiny"])
+    r = O.beam_step(x.hidden, x.w_vocab, x.token_ids, x.block_offsets, x.cand_offsets, x.draft_tok_logprob,
+                    x.reward, 1.0, x.uniforms, 0.7)
+    for key in ("tok_logprob", "blk_logprob", "weights"):
+        want = np.array([float.fromhex(v) for v in stored[key]])
+        assert np.allclose(r[key], want, rtol=1e-12, atol=1e-13), key     # BLAS summation order may differ between hosts
+    assert [int(v) for v in stored["chosen"]] == r["chosen"].tolist()
+    assert [int(v) for v in stored["accept"]] == r["accept"].tolist()
