@@ -819,3 +819,39 @@ def test_random_shapes_against_the_oracle(ctx, d, V, P, n, lo, hi, mode):
     for key in ("tok_logprob", "blk_logprob_f64", "blk_logprob_gen", "weights", "chosen", "accept"):
         assert np.array_equal(fused[key], sep[key]), key
     assert ctx.device_status() == 0
+
+
+# ------------------------------------------------------------------------------- argument checks of the wider API
+
+def test_argument_checks_of_the_dual_shard_and_gather_calls(ctx):
+    cfg = small_config("args2", (4, 4), 1, 2, 64, 300, seed=6200)
+    x = I.make_step_inputs(cfg)
+    s = DeviceStep(ctx, x)
+    dev = "cuda:0"
+    gen_tok = torch.empty(x.rows, dtype=torch.float32, device=dev)
+    ws = torch.empty(ctx.beam_step_dual_workspace_bytes(x.rows, 64, 64, 300), dtype=torch.uint8, device=dev)
+
+    def status_of(fn):
+        with pytest.raises(binding.SpecsError) as e:
+            fn()
+        return e.value.status
+
+    dual = lambda **kw: ctx.specs_beam_step_dual(
+        s.hidden, s.w_vocab, kw.get("h_g", s.hidden), s.w_vocab, s.token_ids, s.block_offsets, s.cand_offsets, s.reward,
+        s.uniforms, 1.0, 0.5, s.tok_lp, kw.get("gen_tok", gen_tok), s.blk_lp64, s.gen_blk64, s.weights, s.chosen,
+        s.accept, kw.get("ws", ws))
+    assert status_of(lambda: dual(gen_tok=None)) == 1             # the generator's log-probs are an output here
+    assert status_of(lambda: dual(ws=ws[:64])) == 4
+    assert status_of(lambda: dual(h_g=s.hidden[:, :12])) == 2     # d_gen % 8 != 0
+    part = torch.empty((x.rows, 4), dtype=torch.float32, device=dev)
+    assert status_of(lambda: ctx.specs_score_partials(s.hidden, s.w_vocab, s.token_ids, -1, part, s.workspace)) == 2
+    assert status_of(lambda: ctx.specs_score_partials(s.hidden, s.w_vocab, None, 0, part, s.workspace)) == 1
+    assert status_of(lambda: ctx.specs_merge_partials(part.view(1, x.rows, 4)[:0], s.token_ids, 300, s.tok_lp)) == 2
+    ids_out = torch.empty((1, 8), dtype=torch.int32, device=dev)
+    len_out = torch.empty(1, dtype=torch.int32, device=dev)
+    assert status_of(lambda: ctx.specs_gather_chosen(s.token_ids, s.block_offsets, s.cand_offsets, s.chosen,
+                                                     ids_out[:, :0], len_out)) == 2
+    assert status_of(lambda: ctx.specs_gather_chosen(s.token_ids, s.block_offsets, s.cand_offsets, None,
+                                                     ids_out, len_out)) == 1
+    torch.cuda.synchronize()
+    assert torch.isnan(s.tok_lp).all() and ctx.device_status() == 0     # nothing was launched
