@@ -855,3 +855,43 @@ def test_argument_checks_of_the_dual_shard_and_gather_calls(ctx):
                                                      ids_out, len_out)) == 1
     torch.cuda.synchronize()
     assert torch.isnan(s.tok_lp).all() and ctx.device_status() == 0     # nothing was launched
+
+
+def test_run_specs_helper_follows_the_controller(ctx):
+    # the packaged loop (controller + fused step + gather) with a stub generator that records what it was asked
+    from paper_2506_15733_b200 import loop as LP
+    P, n, d, Vv = 3, 4, 64, 500
+    w_bits = I.make_step_inputs(small_config("loop_w", (1, 1), 1, 1, d, Vv, seed=5500)).w_vocab
+    w_dev = binding.bf16_bits_to_device(w_bits, "cuda:0")
+    asked, batches = [], []
+
+    def draft_fn(gens, live):
+        asked.append(gens.copy())
+        x = I.make_step_inputs(small_config("loop", (4, 12), len(live), n, d, Vv, seed=6300 + len(asked)))
+        x.w_vocab = w_bits                                 # the same LM head at every step
+        for j, p in enumerate(live):                       # the target's candidates earn higher rewards
+            sl = slice(j * n, (j + 1) * n)
+            x.reward[sl] = np.float32(0.5) + x.reward[sl] / 2 if gens[p] == binding.GEN_TARGET else x.reward[sl] / 2
+        s = DeviceStep(ctx, x)
+        batches.append((x, live.copy()))
+        return LP.DraftBatch(s.hidden, s.token_ids, s.block_offsets, s.cand_offsets, s.reward, s.uniforms, s.draft)
+
+    ctl = binding.Controller(P, binding.POLICY_SPECS, target_len=40)
+    res = LP.run_specs(ctx, ctl, draft_fn, w_dev, 1.0, 0.8, max_block_len=16, max_iters=50)
+    assert (ctl.generators() == binding.GEN_DONE).all()
+    assert all(g[0] == binding.GEN_TARGET for g in res.generators)          # Algorithm 1 begins with the target
+    assert [len(t) for t in res.traces] == res.stats["length"].tolist() and min(res.stats["length"]) >= 40
+    # every appended token is one of the drafted ids of that step, in block order
+    pos = [0] * P
+    for (x, live), gens in zip(batches, asked):
+        ref = oracle_step(x, 1.0, 0.8)
+        for j, p in enumerate(live):
+            a = int(x.cand_offsets[j])
+            lens = np.diff(x.block_offsets)[a:a + n]
+            took = res.traces[p][pos[p]:]
+            match = [c for c in range(n) if took[:lens[c]] == x.token_ids[x.block_offsets[a + c]:x.block_offsets[a + c + 1]].tolist()]
+            assert match, "the appended tokens are not one of the candidates"
+            if ref["margin"][j] > MARGIN + 1e-2:
+                assert int(ref["chosen"][j]) in match
+            pos[p] += int(lens[match[0]]) if int(ref["chosen"][j]) not in match else int(lens[int(ref["chosen"][j])])
+    assert ctx.device_status() == 0
