@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libspecs_b200.so")
-SOURCES = ["api.cu", "score_tcgen05.cu", "score_simt.cu", "select_kernels.cu", "score_noalloc.cu", "controller.cpp"]
+SOURCES = ["api.cu", "planner.cu", "score_tcgen05.cu", "score_simt.cu", "select_kernels.cu", "score_noalloc.cu", "controller.cpp"]
 
 
 def _nvcc() -> str:

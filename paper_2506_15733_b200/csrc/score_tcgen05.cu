@@ -67,6 +67,7 @@
 #include <cuda_bf16.h>
 
 #include <atomic>
+#include <map>
 #include <mutex>
 
 #include "specs_internal.h"
@@ -905,12 +906,11 @@ int launch_wait_expiry_probe(specs_ctx* ctx, unsigned long long limit_ns, cudaSt
 int query_pair_units(int device, int num_sms) {
     // Per device, once: opt both kernels in to their dynamic shared memory (a per-device function
     // attribute) and ask how many CTA pairs the device keeps resident at once.
-    static int cached[64];
-    static bool done[64] = {};
+    static std::map<int, int> cached;                        // device -> resident pairs
     static std::mutex guard;
     std::lock_guard<std::mutex> lock(guard);
-    const int slot = device & 63;
-    if (done[slot]) return cached[slot];
+    const auto hit = cached.find(device);
+    if (hit != cached.end()) return hit->second;
     int units = 0;
     const bool ok1 = cudaFuncSetAttribute(score_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)Shape<1>::kSmemBytes) == cudaSuccess;
@@ -936,8 +936,7 @@ int query_pair_units(int device, int num_sms) {
     }
     cudaGetLastError();                                      // a failed query is not an error of the caller
     if (!ok1) return 0;                                      // try again on the next call
-    cached[slot] = units;
-    done[slot] = true;
+    cached[device] = units;
     return units;
 }
 
