@@ -459,6 +459,8 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
     if (kCg == 2) cluster_sync_all();     // the peer's barriers are initialised before anything reaches them
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&sh->tmem_base);
+    // the kernel may have been launched while its predecessor in the stream still ran: wait for it here
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // Registers move from the control warpgroup (which needs few) to the two epilogue warpgroups
     // (128 fp32 partial logits per thread).  Each setmaxnreg sits at the
@@ -976,18 +978,32 @@ int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan_in, const void* h
         tl = &ctx->timed[ctx->timed_used++];
         cudaEventRecord(tl->start, stream);
     }
+    // Programmatic stream serialisation: the launch is set up, and the CTAs do their prologue (barriers, tensor
+    // memory), while the previous kernel of the stream still runs; griddepcontrol.wait in the kernel orders
+    // everything that touches global memory after that kernel.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)plan.grid, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = pair ? Shape<2>::kSmemBytes : Shape<1>::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t le;
     if (fp8 && pair)
-        score_tiles_pair_fp8_kernel<<<plan.grid, kThreads, Shape<2>::kSmemBytes, stream>>>(
-            map_h, map_w, plan, token_ids, workspace, ctx->d_status, hidden_scale, w_scale);
+        le = cudaLaunchKernelEx(&cfg, score_tiles_pair_fp8_kernel, map_h, map_w, plan, token_ids, workspace,
+                                ctx->d_status, hidden_scale, w_scale);
     else if (fp8)
-        score_tiles_fp8_kernel<<<plan.grid, kThreads, Shape<1>::kSmemBytes, stream>>>(
-            map_h, map_w, plan, token_ids, workspace, ctx->d_status, hidden_scale, w_scale);
+        le = cudaLaunchKernelEx(&cfg, score_tiles_fp8_kernel, map_h, map_w, plan, token_ids, workspace, ctx->d_status,
+                                hidden_scale, w_scale);
     else if (pair)
-        score_tiles_pair_kernel<<<plan.grid, kThreads, Shape<2>::kSmemBytes, stream>>>(map_h, map_w, plan, token_ids,
-                                                                                      workspace, ctx->d_status);
+        le = cudaLaunchKernelEx(&cfg, score_tiles_pair_kernel, map_h, map_w, plan, token_ids, workspace,
+                                ctx->d_status);
     else
-        score_tiles_kernel<<<plan.grid, kThreads, Shape<1>::kSmemBytes, stream>>>(map_h, map_w, plan, token_ids,
-                                                                                 workspace, ctx->d_status);
+        le = cudaLaunchKernelEx(&cfg, score_tiles_kernel, map_h, map_w, plan, token_ids, workspace, ctx->d_status);
+    if (le != cudaSuccess) return SPECS_ERR_CUDA;
     if (tl) cudaEventRecord(tl->stop, stream);
     return cuda_status(cudaGetLastError());
 }

@@ -341,6 +341,8 @@ finish_step_kernel(const ScorePlan plan, const float* __restrict__ workspace, co
                    uint32_t* __restrict__ status) {
     // Launched with programmatic stream serialisation: wait here for the scoring kernel's results.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // let the next kernel of the stream (the next step's scoring kernel) begin its prologue
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int p = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int a = cand_offsets[p], b = cand_offsets[p + 1];
