@@ -37,7 +37,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM bytes (read + write) of one launch of the scoring kernel, from the ncu capture summarised
 # under profiles/ (null until a capture for that workload exists).
-NCU_TRAFFIC_BYTES = {"step7b": 1.1759e9 + 3.8e6}   # profiles/score_tiles_pair_kernel_step7b.md
+NCU_TRAFFIC_BYTES = {"step7b": 1.0995e9 + 3.75e6}   # profiles/score_tiles_pair_kernel_step7b.md
 
 
 def load_peaks():
