@@ -53,7 +53,8 @@ typedef enum specs_status {
 /* Bits of the device status word returned by specs_device_status(). */
 #define SPECS_DEV_TIMEOUT      0x1u
 #define SPECS_DEV_TOKEN_RANGE  0x2u
-#define SPECS_DEV_ACCUM_RANGE  0x4u   /* advisory, see specs_set_accum_chunk; does not change a return value */
+#define SPECS_DEV_ACCUM_RANGE  0x4u   /* informational: some rows were re-scored by the second pass, see
+                                         specs_set_accum_chunk; does not change a return value */
 
 /* Scoring engines (see specs_set_engine). */
 #define SPECS_ENGINE_TCGEN05      0   /* tensor-core path: TMA + tcgen05.mma + TMEM, fused epilogue (default);
@@ -87,18 +88,21 @@ int specs_set_engine(specs_ctx* ctx, int engine);
  *   k_elements > 0 (a multiple of 64): fixed chunks of that length.
  *   k_elements = 0: one accumulator over the whole of d.
  *   SPECS_ACCUM_ADAPTIVE (default): 512-element chunks for the first two vocabulary
- *     tiles of each run of tiles a CTA (pair) scores for its rows; the largest
- *     |logit| of the first tile then sets the chunk length of the remaining tiles:
- *     as many K = 16 accumulations as keep (count x fp32 spacing at twice that
- *     magnitude) below 1e-3, a worst-case figure of which about an eighth is seen
- *     in practice, never shorter than 512 elements.  |logit| below 32 runs d <= 4160
+ *     tiles of each run of tiles a CTA (pair) scores for its rows; the |logit| magnitudes
+ *     of the first tile then set the chunk length of the remaining tiles: as many K = 16
+ *     accumulations as keep (count x fp32 spacing at the magnitude class, a power of
+ *     two, that all but 1/32 of the tile's rows stay within at twice their largest
+ *     |logit|) below 1e-3, a worst-case figure of which about an eighth is seen in
+ *     practice, never shorter than 512 elements.  Magnitudes below 32 run d <= 4160
  *     unchunked, below 64 in 2048-element chunks, ... , from 256 on in 512-element
- *     chunks.  Measured at d = 5120 against the exact result: at most 1.9e-4 per token
- *     for logit spreads up to 48, where a single chunk would be off by 2.3e-3.  If a
- *     later tile of the run holds a positive logit, or the drafted id's logit, beyond
- *     the binade assumed, the results stand but the advisory bit
- *     SPECS_DEV_ACCUM_RANGE is set: those rows may carry a few 1e-3 of accumulation
- *     bias; rescore with a fixed chunk if that matters. */
+ *     chunks.  A row in which a logit that matters (its largest, or the drafted id's)
+ *     turns out to lie beyond that class -- anywhere in the vocabulary, or because the
+ *     row is one of the few far larger than its tile -- is marked, and a second launch
+ *     of the scoring kernel re-scores the marked rows with 512-element chunks (all rows
+ *     when more than about an eighth of them are marked), so the per-token error stays
+ *     within 2e-3 whatever the data; SPECS_DEV_ACCUM_RANGE then reports that this
+ *     happened.  Measured at d = 5120 against the exact result: at most 1.9e-4 per token
+ *     for logit spreads up to 48, where a single chunk would be off by 2.3e-3. */
 #define SPECS_ACCUM_ADAPTIVE (-1)
 int specs_set_accum_chunk(specs_ctx* ctx, int32_t k_elements);
 
@@ -116,8 +120,11 @@ int specs_sm_count(const specs_ctx* ctx);
 
 /* Bytes of scratch specs_score_blocks needs for these sizes.  It holds one
  * (running max, sum of exponentials, drafted-token logit) triple per row and per
- * vocabulary split -- a few hundred KB per 148 row tiles -- and never anything
- * proportional to rows x V: the logits themselves exist only in tensor memory. */
+ * vocabulary split -- a few hundred KB per 148 row tiles -- twice (for the two
+ * scoring passes of adaptive accumulation chunks), and a buffer for the hidden
+ * states of the rows the second pass re-scores (an eighth of the rows, 8192 at
+ * most); never anything proportional to rows x V: the logits themselves exist only
+ * in tensor memory. */
 size_t specs_score_workspace_bytes(const specs_ctx* ctx, int64_t rows, int32_t d, int32_t V);
 
 /* log pi_target of every drafted token and of every drafted block
@@ -242,11 +249,13 @@ int specs_prm_rewards(specs_ctx* ctx, const void* prm_hidden, const int64_t* blo
 int specs_accept(specs_ctx* ctx, const float* reward, const int32_t* cand_offsets, int32_t P,
                  float tau, uint8_t* accept, void* cuda_stream);
 
-/* One whole beam step on DEVICE buffers in two launches: the LM-head scoring
- * kernel, then one kernel that, per problem, merges the vocabulary splits into
- * log pi_target of every drafted token (Section 2, Appendix E.3), sums target and
- * generator log-probabilities per drafted block (Eq. 1), draws SubSample's
- * candidate (Algorithm 2) and evaluates the switch test (Algorithm 1, Step III).
+/* One whole beam step on DEVICE buffers, as one chain of launches that overlap
+ * their set-up with their predecessors: the LM-head scoring kernel, the merge of its
+ * vocabulary splits into log pi_target of every drafted token (Section 2, Appendix
+ * E.3), the second scoring pass (with adaptive chunks; it returns at once when no row
+ * was marked), and one kernel that, per problem, sums target and generator
+ * log-probabilities per drafted block (Eq. 1), draws SubSample's candidate
+ * (Algorithm 2) and evaluates the switch test (Algorithm 1, Step III).
  * Results are identical to specs_score_blocks + specs_block_sums +
  * specs_subsample_f64 on the same inputs; only the launch count differs.
  *
@@ -273,10 +282,10 @@ int specs_beam_step(specs_ctx* ctx, const void* hidden, const void* W_vocab, con
  * given: the drafted tokens are scored with the generator's own LM head as well
  * (its final hidden states hidden_gen [rows, d_gen] and weights W_gen [V, d_gen];
  * Appendix E.1 lists scoring with the draft and with the target model), and Eq. (1)
- * takes the two block log-probabilities.  Three launches: the generator-shaped
- * scoring pass, the target-shaped one, and one finish kernel that merges both,
- * writes both per-token log-probabilities (their difference is the per-token
- * log-ratio), sums them per block, runs SubSample and the switch test and, when
+ * takes the two block log-probabilities.  The generator-shaped head is scored first
+ * (scoring kernel, merge, second pass), then the target-shaped one, and one finish
+ * kernel sums both per-token log-probabilities (their difference is the per-token
+ * log-ratio) per block, runs SubSample and the switch test and, when
  * chosen_ids is given, gathers the selected block's token ids for the append of
  * Algorithm 1, Step II (see specs_gather_chosen).
  *
@@ -454,14 +463,15 @@ int specs_beam_step_host(specs_ctx* ctx,
  * counterpart; it is how the expiry path is tested without a stuck GPU.) */
 int specs_probe_wait_expiry(specs_ctx* ctx, int64_t limit_us, void* cuda_stream);
 
-/* Per-launch timing of the tensor-core scoring kernel.  specs_set_timing(ctx, 1)
+/* Per-call timing of the tensor-core scoring kernel.  specs_set_timing(ctx, 1)
  * makes every later scoring call on this context record a CUDA event before and
- * after that kernel on the call's own stream (a few microseconds each; off by
- * default) and forgets earlier records; (ctx, 0) stops recording and keeps the
+ * after each launch of that kernel on the call's own stream (a few microseconds each;
+ * off by default) and forgets earlier records; (ctx, 0) stops recording and keeps the
  * records; (ctx, 2) resumes recording without forgetting, so that a caller can
- * time every K-th launch of a loop.  specs_score_kernel_ms() waits for the recorded
- * launches, returns their MEAN duration in milliseconds, stores their number in
- * *h_launches (may be NULL) and forgets them; it returns a negative value when
+ * time every K-th call of a loop.  specs_score_kernel_ms() waits for the recorded
+ * launches, returns the MEAN duration per scoring call in milliseconds (its pass over
+ * all rows plus its second pass over re-scored rows), stores the number of calls in
+ * *h_launches (may be NULL) and forgets the records; it returns a negative value when
  * nothing was recorded. */
 int   specs_set_timing(specs_ctx* ctx, int enabled);
 float specs_score_kernel_ms(specs_ctx* ctx, int32_t* h_launches);
@@ -497,8 +507,10 @@ int specs_score_plan_unit(int64_t rows, int32_t d, int32_t V, int32_t num_sms, i
  * which every GPU that loads the library holds until the process exits.  The call
  * itself, and everything it runs, calls no cudaMalloc, cudaFree or other allocating
  * routine; inputs and outputs are the caller's buffers as in specs_score_blocks
- * (same meaning, layout and requirements), always on the tensor-core engine, on the
- * CURRENT device.
+ * (same meaning, layout and requirements), always on the tensor-core engine with
+ * fixed 512-element accumulation chunks (the adaptive chunks of the regular entry
+ * point need a second pass and a buffer of gathered rows, which would not fit), on
+ * the CURRENT device.
  *
  *   status_word  device uint32 that receives SPECS_DEV_* bits by atomic OR (never
  *                cleared by the library); NULL sends them to an internal word that
@@ -507,7 +519,7 @@ int specs_score_plan_unit(int64_t rows, int32_t d, int32_t V, int32_t num_sms, i
  * Limits and sharing:
  *   - the plan for (rows, d, V) must fit the fixed scratch (waves x SMs x 3072 bytes
  *     <= SPECS_NOALLOC_SCRATCH_BYTES; roughly 50 000 rows at d = 3584 or 5120 and
- *     170 000 at d = 1536 on a 148-SM part; specs_score_plan gives the exact size);
+ *     170 000 at d = 1536 on a 148-SM part: waves and CTAs as specs_score_plan reports them);
  *     larger problems return SPECS_ERR_LIMIT and launch nothing.  Split the rows over
  *     several calls instead.
  *   - all calls on a device share the one array, which still holds the previous

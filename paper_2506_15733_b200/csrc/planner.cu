@@ -86,7 +86,7 @@ ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, i
 }
 
 size_t plan_workspace_bytes(const ScorePlan& p) {
-    return plan_slot_bytes(p) + (size_t)p.units * sizeof(uint64_t);
+    return plan_layout(p).total;
 }
 
 }  // namespace specs

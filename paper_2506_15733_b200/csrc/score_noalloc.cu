@@ -91,7 +91,10 @@ extern "C" int specs_score_blocks_noalloc(const void* hidden, const void* W_voca
     int st = setup_current_device(device, &setup);
     if (st != SPECS_OK) return st;
 
-    const specs::ScorePlan plan = specs::make_score_plan(rows, d, V, setup.num_sms, setup.pair_units);
+    // Fixed 512-element accumulation chunks: exact enough for any logit magnitude without the second
+    // pass (and the buffer of gathered rows) that adaptive chunks need, so the scratch stays small.
+    const specs::ScorePlan plan = specs::make_score_plan(rows, d, V, setup.num_sms, setup.pair_units,
+                                                         specs::kCtaGroupAuto, specs::kDefaultChunkKBlocks, false);
     if (specs::plan_workspace_bytes(plan) > (size_t)SPECS_NOALLOC_SCRATCH_BYTES) return SPECS_ERR_LIMIT;
 
     // A context that lives on this stack frame only: it carries what the launchers read
@@ -105,10 +108,10 @@ extern "C" int specs_score_blocks_noalloc(const void* hidden, const void* W_voca
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
     if (rows > 0) {
-        float* scratch = static_cast<float*>(setup.scratch);
+        void* scratch = setup.scratch;
         st = specs::launch_score_tcgen05(&local, plan, hidden, W_vocab, token_ids, scratch, stream);
         if (st != SPECS_OK) return st;
-        st = specs::launch_merge(&local, plan, scratch, token_ids, tok_logprob, stream);
+        st = specs::launch_merge(&local, plan, scratch, token_ids, tok_logprob, nullptr, hidden, nullptr, stream);
         if (st != SPECS_OK) return st;
     }
     if (B > 0 && (blk_logprob || blk_logprob_f64))

@@ -171,8 +171,8 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
         : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ void st_cluster_f32(uint32_t cluster_addr, float v) {
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v) : "memory");
+__device__ __forceinline__ void st_cluster_u64(uint32_t cluster_addr, uint64_t v) {
+    asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(cluster_addr), "l"(v) : "memory");
 }
 
 // The abort flag of this CTA and, in the pair kernel, the shared::cluster address of the
@@ -358,52 +358,92 @@ struct SharedLayout {
     uint64_t empty[kMaxStages];  // MMA -> TMA: stage may be overwritten
     uint64_t acc_full[2];        // MMA -> epilogue: accumulator complete
     uint64_t acc_empty[2];       // epilogue -> MMA: accumulator drained (pair: only the leader's is used)
-    uint64_t mode;               // epilogue warps -> MMA issuer and epilogue: |logit| maxima published
-    float absmax[2 * kEpilogueWarps];   // largest |logit| of the run's first tile, per epilogue warp of the unit
+    uint64_t mode;               // epilogue warps -> MMA issuer and epilogue: magnitude counts published
+    uint64_t mag_counts[2 * kEpilogueWarps];   // per epilogue warp of the unit: see pack_magnitude_counts
+    ScorePlan plan2;             // second pass: the plan derived from the number of marked rows
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
 
-// Chunk length (in k-blocks) for logits whose magnitude stays below twice `absmax`.
-// One accumulation (one MMA instruction along K) truncates the fp32 accumulator toward zero by at most
-// one spacing of its magnitude.  The chunk gets as many accumulations as keep (count x spacing at twice
-// the sampled magnitude) under 1e-3, half of the 2e-3 tolerance on a token log-probability.  That product
-// is a worst case: the loss per accumulation averages half a spacing, and of the partial sum's magnitude,
-// not the final one's; measured, the bias is about a quarter of it (-5e-3 at |logit| = 700, d = 5120,
-// one chunk: bound 2e-2), and another factor of two is the margin on the sampled magnitude.  The chunk is
-// never shorter than `base`.  `*bound` receives the magnitude up to which that spacing holds (the top of
-// the binade).
-__device__ __forceinline__ int adaptive_chunk_kblocks(float absmax, int base, int k_blocks, float* bound) {
-    *bound = INFINITY;                                       // no claim when the base chunk is kept
+// Magnitude class of a thread's largest |logit| in the run's first tile: the e with max(2 |logit|, 1) in
+// [2^(e-1), 2^e), 1..10; 11 from 1024 on (and for NaN).  The factor two is margin: the maximum over the
+// whole vocabulary lies above the maximum over one tile.
+__device__ __forceinline__ int magnitude_class(float absmax) {
     const float a = fmaxf(2.0f * absmax, 1.0f);
-    if (!(a < 1024.0f)) return base;                         // also NaN and inf
-    const int e = ((__float_as_int(a) >> 23) & 0xff) - 126;  // a = m * 2^e with m in [0.5, 1)
-    const float n_acc = ldexpf(1.0e-3f, 24 - e);             // spacing of [2^(e-1), 2^e) is 2^(e-24)
-    int kb = (int)(n_acc * 0.25f);                           // four accumulations per k-block
+    if (!(a < 1024.0f)) return 11;
+    return ((__float_as_int(a) >> 23) & 0xff) - 126;         // a = m * 2^e with m in [0.5, 1)
+}
+// One word per warp: for t = 1..10, six bits holding how many of the warp's lanes have a class above t.
+__device__ __forceinline__ uint64_t pack_magnitude_counts(int cls) {
+    uint64_t w = 0;
+#pragma unroll
+    for (int t = 1; t <= 10; ++t)
+        w |= (uint64_t)__popc(__ballot_sync(0xffffffffu, cls > t)) << (6 * (t - 1));
+    return w;
+}
+// The class the unit's chunks are sized for: the smallest one that all but 1/32 of the unit's (row, column
+// half) samples stay within.  A few rows with far larger logits than the rest (which the merge will send to
+// the second pass anyway) therefore do not shorten the chunks of their whole tile.
+template <int kCg>
+__device__ __forceinline__ int read_magnitude_class(const SharedLayout* sh) {
+    const volatile uint64_t* p = sh->mag_counts;
+    uint32_t above[10];
+#pragma unroll
+    for (int t = 0; t < 10; ++t) above[t] = 0;
+#pragma unroll
+    for (int i = 0; i < kEpilogueWarps * kCg; ++i) {
+        const uint64_t w = p[i];
+#pragma unroll
+        for (int t = 0; t < 10; ++t) above[t] += (uint32_t)(w >> (6 * t)) & 63u;
+    }
+    constexpr uint32_t kBudget = 8 * kCg;                    // of 256 * kCg samples
+    int cls = 11;
+#pragma unroll
+    for (int t = 9; t >= 0; --t) cls = (above[t] <= kBudget) ? t + 1 : cls;
+    return cls;
+}
+
+// Chunk length (in k-blocks) for logits of magnitude class `cls`, i.e. below 2^cls.
+// One accumulation (one MMA instruction along K) truncates the fp32 accumulator toward zero by at most
+// one spacing of its magnitude.  The chunk gets as many accumulations as keep (count x spacing below 2^cls)
+// under 1e-3, half of the 2e-3 tolerance on a token log-probability.  That product is a worst case: the
+// loss per accumulation averages half a spacing, and of the partial sum's magnitude, not the final one's;
+// measured, the bias is about a quarter of it (-5e-3 at |logit| = 700, d = 5120, one chunk: bound 2e-2).
+// The chunk is never shorter than `base`.  `*bound` receives the magnitude up to which that holds (2^cls),
+// infinity when the base chunk is kept: nothing shorter exists, so there is nothing to re-score with.
+__device__ __forceinline__ int adaptive_chunk_kblocks(int cls, int base, int k_blocks, float* bound) {
+    *bound = INFINITY;
+    if (cls > 10) return base;
+    const float n_acc = ldexpf(1.0e-3f, 24 - cls);           // spacing of [2^(cls-1), 2^cls) is 2^(cls-24)
+    int kb = (int)fminf(n_acc * 0.25f, 1.0e6f);              // four accumulations per k-block
     if (kb <= base) return base;
-    *bound = ldexpf(1.0f, e);
+    *bound = ldexpf(1.0f, cls);
     if (kb >= k_blocks) return k_blocks;
     const int chunks = (k_blocks + kb - 1) / kb;             // equal chunks
     return (k_blocks + chunks - 1) / chunks;
 }
-// Largest published maximum of the unit (8 values per CTA of the unit).
-template <int kCg>
-__device__ __forceinline__ float read_absmax(const SharedLayout* sh) {
-    const volatile float* p = sh->absmax;
-    float m = 0.0f;
-#pragma unroll
-    for (int i = 0; i < kEpilogueWarps * kCg; ++i) m = fmaxf(m, p[i]);
-    return m;
-}
+
+// What links the two passes of an adaptive plan (see FixCtl): the first pass resets the count of marked
+// rows; the second reads it, the list of marked rows and, for 8-bit operands, their gathered scales.
+struct PassArgs {
+    FixCtl* ctl;
+    const int32_t* list;
+    const float* scale_compact;
+    int32_t cap_rows;
+};
 
 // kFp8: operands are E4M3 codes (128 elements per 128-byte k-block, K = 32 per MMA) and the epilogue
 // multiplies every accumulator by hidden_scale[row] * w_scale[column] before anything else.
-template <int kCg, bool kFp8>
-__device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, const CUtensorMap& map_w,
-                                                 const ScorePlan& plan, const int32_t* __restrict__ token_ids,
+// kSecond: the second pass.  It returns at once when no row was marked; otherwise it scores, with the base
+// chunks, either the marked rows gathered in the compact buffer (map_compact, plan derived from their
+// number) or, when they outnumber that buffer, every row in place (map_hidden, the first pass's plan).
+template <int kCg, bool kFp8, bool kSecond>
+__device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, const CUtensorMap& map_compact,
+                                                 const CUtensorMap& map_w, const ScorePlan& plan_in,
+                                                 const int32_t* __restrict__ token_ids,
                                                  float* __restrict__ workspace, uint32_t* __restrict__ status,
                                                  const float* __restrict__ hidden_scale,
-                                                 const float* __restrict__ w_scale) {
+                                                 const float* __restrict__ w_scale, const PassArgs pass) {
     constexpr int kElemsK = kFp8 ? 2 * kBlockK : kBlockK;    // elements in a 128-byte k-block
     using S = Shape<kCg>;
     constexpr int kStages = S::kStages;
@@ -426,6 +466,18 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
     AbortFlags ab;
     ab.own = &sh->abort_flag;
     ab.peer = (kCg == 2) ? mapa_shared(smem_u32(&sh->abort_flag), rank ^ 1u) : 0u;
+
+    bool compact = false;                                    // second pass: gathered rows rather than all rows
+    if (kSecond) {
+        // the count is the merge kernel's: wait for it before anything else, and leave when there is no work
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        const uint32_t marked = *reinterpret_cast<const volatile uint32_t*>(&pass.ctl->count);
+        if (marked == 0u) return;                            // every CTA of the grid takes the same decision
+        compact = marked <= (uint32_t)pass.cap_rows;
+        if (threadIdx.x == 0)
+            sh->plan2 = compact ? make_compact_plan(plan_in, (int64_t)marked) : make_inplace_fix_plan(plan_in);
+    }
+    const ScorePlan& plan = kSecond ? sh->plan2 : plan_in;   // (plan2 is read after the barrier below)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -459,8 +511,11 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
     if (kCg == 2) cluster_sync_all();     // the peer's barriers are initialised before anything reaches them
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&sh->tmem_base);
-    // the kernel may have been launched while its predecessor in the stream still ran: wait for it here
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (!kSecond) {
+        // the kernel may have been launched while its predecessor in the stream still ran: wait for it here
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (pass.ctl != nullptr && blockIdx.x == 0 && threadIdx.x == 0) pass.ctl->count = 0u;
+    }
 
     // Registers move from the control warpgroup (which needs few) to the two epilogue warpgroups
     // (128 fp32 partial logits per thread).  Each setmaxnreg sits at the
@@ -480,6 +535,7 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
         uint32_t stage = 0, phase = 0;           // meaningful in lane 0 only
         uint32_t issued = 0;
         bool ok = true;                          // warp-uniform
+        const CUtensorMap* map_rows = (kSecond && compact) ? &map_compact : &map_hidden;
         for (int w = 0; w < plan.waves && ok; ++w) {
             int st, nb, ne;
             if (!plan_unit(plan, w, unit, &st, &nb, &ne)) continue;
@@ -527,12 +583,12 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                         const uint32_t bar = full0 + stage * 8u;
                         if (kCg == 1) {
                             mbar_arrive_expect_tx(bar, kStageBytes);
-                            tma_load_2d(a_dst, &map_hidden, kb * kElemsK, row0, bar);
+                            tma_load_2d(a_dst, map_rows, kb * kElemsK, row0, bar);
                             tma_load_2d(a_dst + kABytes, &map_w, kb * kElemsK, wrow0, bar);
                         } else {
                             // the leader expects both CTAs' bytes; the peer's may be counted first
                             if (rank == 0) mbar_arrive_expect_tx(smem_u32(&sh->full[stage]), 2u * kStageBytes);
-                            tma_load_2d_pair(a_dst, &map_hidden, kb * kElemsK, row0, bar);
+                            tma_load_2d_pair(a_dst, map_rows, kb * kElemsK, row0, bar);
                             tma_load_2d_pair(a_dst + kABytes, &map_w, kb * kElemsK, wrow0, bar);
                         }
                         ++issued;
@@ -587,7 +643,8 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                         }
                         ++mode_runs;
                         float bound;
-                        ck = adaptive_chunk_kblocks(read_absmax<kCg>(sh), plan.chunk_kblocks, plan.k_blocks, &bound);
+                        ck = adaptive_chunk_kblocks(read_magnitude_class<kCg>(sh), plan.chunk_kblocks, plan.k_blocks,
+                                                    &bound);
                     }
                     for (int kb0 = 0; kb0 < plan.k_blocks && ok; kb0 += ck, ++chunk_count) {
                         const uint32_t buf = chunk_count & 1u;
@@ -655,9 +712,12 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
             int ck = plan.chunk_kblocks;                     // k-blocks per chunk of the current tile
             float assumed = INFINITY;                        // magnitude the lengthened chunks were sized for
             const int64_t row = (int64_t)(st * kCg + (int)rank) * kBlockM + row_in_tile;
+            // the row of the caller's arrays behind this one: itself, or the marked row gathered here
+            const int64_t src = (kSecond && compact && row < plan.rows) ? (int64_t)pass.list[row] : row;
             // ids are indices into the whole vocabulary; this W holds rows id_offset .. id_offset + V - 1
-            const int32_t id = (row < plan.rows) ? token_ids[row] - plan.id_offset : -1;
-            const float row_scale = (kFp8 && row < plan.rows) ? hidden_scale[row] : 0.0f;
+            const int32_t id = (row < plan.rows) ? token_ids[src] - plan.id_offset : -1;
+            float row_scale = 0.0f;
+            if (kFp8 && row < plan.rows) row_scale = (kSecond && compact) ? pass.scale_compact[row] : hidden_scale[src];
             // state in base-2 units: run_max = max(z) * log2(e), run_sum = sum 2^(z*log2e - run_max)
             float run_max = -INFINITY, run_sum = 0.0f, picked = -INFINITY;
             for (int n = nb; n < ne && ok; ++n) {
@@ -668,7 +728,8 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                         break;
                     }
                     ++mode_runs;
-                    ck = adaptive_chunk_kblocks(read_absmax<kCg>(sh), plan.chunk_kblocks, plan.k_blocks, &assumed);
+                    ck = adaptive_chunk_kblocks(read_magnitude_class<kCg>(sh), plan.chunk_kblocks, plan.k_blocks,
+                                                &assumed);
                 }
                 float acc[kHalfN];                           // this thread's 128 logits of the tile
                 for (int kb0 = 0; kb0 < plan.k_blocks; kb0 += ck, ++chunk_count) {
@@ -719,22 +780,22 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                     }
                 }
                 if (adapt_run && n == nb) {
-                    // first tile of the run: publish this warp's largest |logit| to every CTA of the unit
+                    // first tile of the run: publish how this warp's rows are spread over the magnitude classes
+                    // to every CTA of the unit
                     float amax = 0.0f;
 #pragma unroll
                     for (int j = 0; j < kHalfN; ++j)
                         amax = (col_base + j < plan.V) ? fmaxf(amax, fabsf(acc[j])) : amax;
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+                    const uint64_t counts = pack_magnitude_counts(magnitude_class(amax));
                     if (lane == 0) {
                         const int slot = (int)rank * kEpilogueWarps + (warp - 4);
                         if (kCg == 1) {
-                            sh->absmax[slot] = amax;
+                            *reinterpret_cast<volatile uint64_t*>(&sh->mag_counts[slot]) = counts;
                             mbar_arrive(smem_u32(&sh->mode));
                         } else {
 #pragma unroll
                             for (uint32_t r = 0; r < 2; ++r) {
-                                st_cluster_f32(mapa_shared(smem_u32(&sh->absmax[slot]), r), amax);
+                                st_cluster_u64(mapa_shared(smem_u32(&sh->mag_counts[slot]), r), counts);
                                 mbar_arrive_cluster(mapa_shared(smem_u32(&sh->mode), r));
                             }
                         }
@@ -772,12 +833,15 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                 }
             }
             if (ok) {
-                // a positive logit or the drafted id's logit beyond the magnitude the chunks were sized for
-                if (run_max > assumed * kLog2e || (picked != -INFINITY && fabsf(picked) > assumed))
-                    atomicOr(status, SPECS_DEV_ACCUM_RANGE);
+                // A logit that matters -- this part's maximum (the terms of the sum that count lie next to it)
+                // or the drafted id's -- beyond the magnitude the lengthened chunks were sized for: the row is
+                // marked by the sign of its sum (which is positive otherwise) and re-scored in the second pass.
+                const bool over = run_sum > 0.0f && (fabsf(run_max) > assumed * kLog2e ||
+                                                     (picked != -INFINITY && fabsf(picked) > assumed));
+                if (__any_sync(0xffffffffu, over) && lane == 0) atomicOr(status, SPECS_DEV_ACCUM_RANGE);
                 float* slot = workspace + ((size_t)w * plan.grid + cta) * kTripleFloats + half * 3 * kBlockM;
                 slot[row_in_tile] = run_max;
-                slot[kBlockM + row_in_tile] = run_sum;
+                slot[kBlockM + row_in_tile] = over ? -run_sum : run_sum;
                 slot[2 * kBlockM + row_in_tile] = picked;
             }
         }
@@ -798,35 +862,37 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
-score_tiles_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_w,
-                   const ScorePlan plan, const int32_t* __restrict__ token_ids,
-                   float* __restrict__ workspace, uint32_t* __restrict__ status) {
-    score_tiles_body<1, false>(map_hidden, map_w, plan, token_ids, workspace, status, nullptr, nullptr);
-}
+// The kernels: {one CTA, CTA pair} x {bf16, E4M3} x {first pass, second pass}, one body.
+#define SPECS_SCORE_KERNEL(name, cluster_attr, kCg, kFp8, kSecond)                                                  \
+    __global__ void cluster_attr __launch_bounds__(kThreads, 1)                                                     \
+    name(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_compact,           \
+         const __grid_constant__ CUtensorMap map_w, const ScorePlan plan, const int32_t* __restrict__ token_ids,    \
+         float* __restrict__ workspace, uint32_t* __restrict__ status, const float* __restrict__ hidden_scale,      \
+         const float* __restrict__ w_scale, const PassArgs pass) {                                                  \
+        score_tiles_body<kCg, kFp8, kSecond>(map_hidden, map_compact, map_w, plan, token_ids, workspace, status,    \
+                                             hidden_scale, w_scale, pass);                                          \
+    }
+#define SPECS_NO_CLUSTER
+SPECS_SCORE_KERNEL(score_tiles_kernel, SPECS_NO_CLUSTER, 1, false, false)
+SPECS_SCORE_KERNEL(score_tiles_pair_kernel, __cluster_dims__(2, 1, 1), 2, false, false)
+SPECS_SCORE_KERNEL(score_tiles_fp8_kernel, SPECS_NO_CLUSTER, 1, true, false)
+SPECS_SCORE_KERNEL(score_tiles_pair_fp8_kernel, __cluster_dims__(2, 1, 1), 2, true, false)
+SPECS_SCORE_KERNEL(score_tiles_second_kernel, SPECS_NO_CLUSTER, 1, false, true)
+SPECS_SCORE_KERNEL(score_tiles_pair_second_kernel, __cluster_dims__(2, 1, 1), 2, false, true)
+SPECS_SCORE_KERNEL(score_tiles_fp8_second_kernel, SPECS_NO_CLUSTER, 1, true, true)
+SPECS_SCORE_KERNEL(score_tiles_pair_fp8_second_kernel, __cluster_dims__(2, 1, 1), 2, true, true)
+#undef SPECS_NO_CLUSTER
+#undef SPECS_SCORE_KERNEL
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-score_tiles_pair_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_w,
-                        const ScorePlan plan, const int32_t* __restrict__ token_ids,
-                        float* __restrict__ workspace, uint32_t* __restrict__ status) {
-    score_tiles_body<2, false>(map_hidden, map_w, plan, token_ids, workspace, status, nullptr, nullptr);
-}
-
-// The same two kernels on E4M3 codes with per-row scales.
-__global__ void __launch_bounds__(kThreads, 1)
-score_tiles_fp8_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_w,
-                       const ScorePlan plan, const int32_t* __restrict__ token_ids, float* __restrict__ workspace,
-                       uint32_t* __restrict__ status, const float* __restrict__ hidden_scale,
-                       const float* __restrict__ w_scale) {
-    score_tiles_body<1, true>(map_hidden, map_w, plan, token_ids, workspace, status, hidden_scale, w_scale);
-}
-
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-score_tiles_pair_fp8_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_w,
-                            const ScorePlan plan, const int32_t* __restrict__ token_ids,
-                            float* __restrict__ workspace, uint32_t* __restrict__ status,
-                            const float* __restrict__ hidden_scale, const float* __restrict__ w_scale) {
-    score_tiles_body<2, true>(map_hidden, map_w, plan, token_ids, workspace, status, hidden_scale, w_scale);
+using ScoreKernel = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const ScorePlan, const int32_t*,
+                             float*, uint32_t*, const float*, const float*, const PassArgs);
+ScoreKernel score_kernel_for(bool pair, bool fp8, bool second) {
+    if (second) {
+        if (fp8) return pair ? score_tiles_pair_fp8_second_kernel : score_tiles_fp8_second_kernel;
+        return pair ? score_tiles_pair_second_kernel : score_tiles_second_kernel;
+    }
+    if (fp8) return pair ? score_tiles_pair_fp8_kernel : score_tiles_fp8_kernel;
+    return pair ? score_tiles_pair_kernel : score_tiles_kernel;
 }
 
 // Row-wise quantisation to E4M3: one warp per row.  scale = absmax / 448; code = nearest E4M3 of
@@ -876,8 +942,16 @@ __global__ void wait_expiry_probe_kernel(unsigned long long limit_ns, uint32_t* 
     if (threadIdx.x == 0 && (!completed || abort_flag != 0u)) atomicOr(status, SPECS_DEV_TIMEOUT);
 }
 
+// Tensor map of a row-major [outer, inner] matrix with 128-byte-swizzled boxes; maps the context has
+// encoded before are found again by what they describe (the weight's map is the same at every call).
 int encode_rows_2d(specs_ctx* ctx, CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer,
                    uint32_t box_inner, uint32_t box_outer, int elem_bytes) {
+    for (const CachedMap& c : ctx->maps)
+        if (c.base == base && c.inner == inner && c.outer == outer && c.box_inner == box_inner &&
+            c.box_outer == box_outer && c.elem_bytes == elem_bytes) {
+            *map = c.map;
+            return SPECS_OK;
+        }
     const cuuint64_t dims[2] = {inner, outer};
     const cuuint64_t strides[1] = {inner * (uint64_t)elem_bytes};   // bytes between consecutive rows
     const cuuint32_t box[2] = {box_inner, box_outer};
@@ -887,7 +961,15 @@ int encode_rows_2d(specs_ctx* ctx, CUtensorMap* map, const void* base, uint64_t 
                                          strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? SPECS_OK : SPECS_ERR_CUDA;
+    if (r != CUDA_SUCCESS) return SPECS_ERR_CUDA;
+    const CachedMap entry = {base, inner, outer, box_inner, box_outer, elem_bytes, *map};
+    if (ctx->maps.size() < kMapCacheSize) {
+        ctx->maps.push_back(entry);
+    } else {
+        ctx->maps[ctx->maps_next] = entry;
+        ctx->maps_next = (ctx->maps_next + 1) % kMapCacheSize;
+    }
+    return SPECS_OK;
 }
 
 }  // namespace
@@ -906,7 +988,7 @@ int launch_wait_expiry_probe(specs_ctx* ctx, unsigned long long limit_ns, cudaSt
 }
 
 int query_pair_units(int device, int num_sms) {
-    // Per device, once: opt both kernels in to their dynamic shared memory (a per-device function
+    // Per device, once: opt the kernels in to their dynamic shared memory (a per-device function
     // attribute) and ask how many CTA pairs the device keeps resident at once.
     static std::map<int, int> cached;                        // device -> resident pairs
     static std::mutex guard;
@@ -914,14 +996,16 @@ int query_pair_units(int device, int num_sms) {
     const auto hit = cached.find(device);
     if (hit != cached.end()) return hit->second;
     int units = 0;
-    const bool ok1 = cudaFuncSetAttribute(score_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)Shape<1>::kSmemBytes) == cudaSuccess;
-    const bool ok2 = cudaFuncSetAttribute(score_tiles_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)Shape<2>::kSmemBytes) == cudaSuccess &&
-                     cudaFuncSetAttribute(score_tiles_pair_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)Shape<2>::kSmemBytes) == cudaSuccess;
-    cudaFuncSetAttribute(score_tiles_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                         (int)Shape<1>::kSmemBytes);
+    bool ok1 = true, ok2 = true;
+    for (int fp8 = 0; fp8 < 2; ++fp8)
+        for (int second = 0; second < 2; ++second) {
+            ok1 = ok1 && cudaFuncSetAttribute(score_kernel_for(false, fp8, second),
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)Shape<1>::kSmemBytes) == cudaSuccess;
+            ok2 = ok2 && cudaFuncSetAttribute(score_kernel_for(true, fp8, second),
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)Shape<2>::kSmemBytes) == cudaSuccess;
+        }
     if (ok2) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(num_sms & ~1), 1, 1);
@@ -942,30 +1026,50 @@ int query_pair_units(int device, int num_sms) {
     return units;
 }
 
-int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan_in, const void* hidden, const void* w_vocab,
-                         const int32_t* token_ids, float* workspace, cudaStream_t stream, int32_t id_offset,
-                         const float* hidden_scale, const float* w_scale) {
+namespace {
+
+// One launch of the scoring kernel: the first pass over all rows, or the second over the marked ones.
+int launch_score_pass(specs_ctx* ctx, const ScorePlan& plan_in, bool second, const void* hidden, const void* w_vocab,
+                      const int32_t* token_ids, void* workspace, cudaStream_t stream, int32_t id_offset,
+                      const float* hidden_scale, const float* w_scale) {
     static_assert(Shape<1>::kSmemBytes <= 227 * 1024 && Shape<2>::kSmemBytes <= 227 * 1024, "shared memory budget");
     static_assert(Shape<1>::kStages <= kMaxStages && Shape<2>::kStages <= kMaxStages, "barrier arrays");
     static_assert(sizeof(SharedLayout) <= 512, "barrier block");
     const bool pair = plan_in.cta_group == 2;
     if (pair && (plan_in.units > ctx->pair_units || (plan_in.grid & 1))) return SPECS_ERR_CUDA;
+    if (second && !plan_in.adaptive) return SPECS_OK;        // only adaptive plans mark rows
     static std::atomic<uint32_t> launch_counter{0};
     ScorePlan plan = plan_in;
     plan.epoch = (launch_counter.fetch_add(1) % 0xfffeu) + 1u;  // never 0
     plan.lead_tiles = ctx->lead_tiles;
     plan.id_offset = id_offset;
     query_pair_units(ctx->device, ctx->num_sms);             // shared-memory opt-in for this device
-    CUtensorMap map_h, map_w;
     const bool fp8 = plan.elem_bytes == 1;
     if (fp8 && (!hidden_scale || !w_scale)) return SPECS_ERR_NULL;
+    const WsLayout lay = plan_layout(plan);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
     const uint32_t box_k = (uint32_t)(kBlockK * 2 / plan.elem_bytes);       // 128 bytes of K
+    CUtensorMap map_h, map_c, map_w;
     int st = encode_rows_2d(ctx, &map_h, hidden, (uint64_t)plan.d, (uint64_t)plan.rows, box_k, kBlockM,
                             plan.elem_bytes);
     if (st != SPECS_OK) return st;
     st = encode_rows_2d(ctx, &map_w, w_vocab, (uint64_t)plan.d, (uint64_t)plan.V, box_k,
                         pair ? Shape<2>::kBRows : Shape<1>::kBRows, plan.elem_bytes);
     if (st != SPECS_OK) return st;
+    map_c = map_h;
+    PassArgs pass = {nullptr, nullptr, nullptr, 0};
+    if (plan.adaptive) {
+        pass.ctl = reinterpret_cast<FixCtl*>(ws + lay.ctl);
+        pass.list = reinterpret_cast<const int32_t*>(ws + lay.list);
+        pass.scale_compact = reinterpret_cast<const float*>(ws + lay.compact_scale);
+        pass.cap_rows = lay.cap_rows;
+        if (second) {
+            st = encode_rows_2d(ctx, &map_c, ws + lay.compact, (uint64_t)plan.d, (uint64_t)lay.cap_rows, box_k,
+                                kBlockM, plan.elem_bytes);
+            if (st != SPECS_OK) return st;
+        }
+    }
+    float* slots = reinterpret_cast<float*>(second ? ws + lay.fix_slots : ws);
 
     TimedLaunch* tl = nullptr;
     if (ctx->timing) {
@@ -976,6 +1080,7 @@ int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan_in, const void* h
             ctx->timed.push_back(t);
         }
         tl = &ctx->timed[ctx->timed_used++];
+        tl->second_pass = second;
         cudaEventRecord(tl->start, stream);
     }
     // Programmatic stream serialisation: the launch is set up, and the CTAs do their prologue (barriers, tensor
@@ -991,21 +1096,39 @@ int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan_in, const void* h
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t le;
-    if (fp8 && pair)
-        le = cudaLaunchKernelEx(&cfg, score_tiles_pair_fp8_kernel, map_h, map_w, plan, token_ids, workspace,
-                                ctx->d_status, hidden_scale, w_scale);
-    else if (fp8)
-        le = cudaLaunchKernelEx(&cfg, score_tiles_fp8_kernel, map_h, map_w, plan, token_ids, workspace, ctx->d_status,
-                                hidden_scale, w_scale);
-    else if (pair)
-        le = cudaLaunchKernelEx(&cfg, score_tiles_pair_kernel, map_h, map_w, plan, token_ids, workspace,
-                                ctx->d_status);
-    else
-        le = cudaLaunchKernelEx(&cfg, score_tiles_kernel, map_h, map_w, plan, token_ids, workspace, ctx->d_status);
+    const cudaError_t le = cudaLaunchKernelEx(&cfg, score_kernel_for(pair, fp8, second), map_h, map_c, map_w, plan,
+                                              token_ids, slots, ctx->d_status, hidden_scale, w_scale, pass);
     if (le != cudaSuccess) return SPECS_ERR_CUDA;
     if (tl) cudaEventRecord(tl->stop, stream);
     return cuda_status(cudaGetLastError());
+}
+
+}  // namespace
+
+int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan, const void* hidden, const void* w_vocab,
+                         const int32_t* token_ids, void* workspace, cudaStream_t stream, int32_t id_offset,
+                         const float* hidden_scale, const float* w_scale) {
+    return launch_score_pass(ctx, plan, false, hidden, w_vocab, token_ids, workspace, stream, id_offset, hidden_scale,
+                             w_scale);
+}
+
+int launch_score_second_pass(specs_ctx* ctx, const ScorePlan& plan, const void* hidden, const void* w_vocab,
+                             const int32_t* token_ids, void* workspace, cudaStream_t stream, int32_t id_offset,
+                             const float* hidden_scale, const float* w_scale) {
+    return launch_score_pass(ctx, plan, true, hidden, w_vocab, token_ids, workspace, stream, id_offset, hidden_scale,
+                             w_scale);
+}
+
+FixView fix_view(const ScorePlan& plan, const void* workspace) {
+    FixView v = {nullptr, nullptr, nullptr, 0};
+    if (!plan.adaptive || workspace == nullptr) return v;
+    const WsLayout lay = plan_layout(plan);
+    const uint8_t* ws = static_cast<const uint8_t*>(workspace);
+    v.ctl = reinterpret_cast<const FixCtl*>(ws + lay.ctl);
+    v.list = reinterpret_cast<const int32_t*>(ws + lay.list);
+    v.slots = reinterpret_cast<const float*>(ws + lay.fix_slots);
+    v.cap_rows = lay.cap_rows;
+    return v;
 }
 
 }  // namespace specs

@@ -7,7 +7,9 @@
 //                         Algorithm 2, a Gumbel-max draw from caller-supplied uniforms and the
 //                         switch test of Algorithm 1, Step III;
 //   accept_kernel         the switch test alone;
-//   finish_step_kernel    all of the above for one problem per CTA, for the fused beam step.
+//   fix_merge_kernel      writes the second scoring pass's results over those of the re-scored rows;
+//   finish_step_kernel    block sums, SubSample and the switch test for one problem per CTA, for the
+//                         fused beam step.
 #include <cuda_bf16.h>
 
 #include "specs_internal.h"
@@ -23,13 +25,15 @@ constexpr unsigned kFull = 0xffffffffu;
 // half of the tile's 256 columns (the two epilogue threads of a row), the running maximum in
 // base-2 units (max logit * log2 e), the sum of 2^(logit*log2e - max) over that half of the CTA's
 // vocabulary chunk, and the drafted id's logit if the id fell there (-inf otherwise).  A half
-// that saw no valid column (vocabulary tail) carries max = -inf, sum = 0.
+// that saw no valid column (vocabulary tail) carries max = -inf, sum = 0.  A NEGATIVE sum is the first
+// pass's mark on a row whose logits outgrew its tile's accumulation chunks: its magnitude is the sum,
+// and the row is re-scored by the second pass.
 constexpr int kMergeBatch = 6;                              // splits whose six floats are loaded before any is used
 
 // Fold of a row's per-split partials, in split order, into (max, sum) in base-2 units and the drafted
 // id's logit.  The loads of a batch of splits are independent of the arithmetic and of each other, so a
 // batch costs one trip to L2.
-struct RowFold { float max2; double sum2; float logit; };
+struct RowFold { float max2; double sum2; float logit; bool marked; };
 
 __device__ __forceinline__ RowFold fold_row(const ScorePlan& plan, const float* __restrict__ workspace, int64_t row) {
     const int mt = (int)(row / kBlockM), r = (int)(row % kBlockM);
@@ -47,7 +51,7 @@ __device__ __forceinline__ RowFold fold_row(const ScorePlan& plan, const float* 
     constexpr int kHalf = 3 * kBlockM;                      // second half of the tile's columns
 
     RowFold f;
-    f.max2 = -INFINITY; f.sum2 = 0.0; f.logit = -INFINITY;
+    f.max2 = -INFINITY; f.sum2 = 0.0; f.logit = -INFINITY; f.marked = false;
     for (int s0 = 0; s0 < splits; s0 += kMergeBatch) {
         float v[kMergeBatch][6];
 #pragma unroll
@@ -56,8 +60,9 @@ __device__ __forceinline__ RowFold fold_row(const ScorePlan& plan, const float* 
             const float* p = base + (size_t)(live ? s0 + u : s0) * stride;
             const float m0 = __ldcg(p), s_0 = __ldcg(p + kBlockM), t0 = __ldcg(p + 2 * kBlockM);
             const float m1 = __ldcg(p + kHalf), s_1 = __ldcg(p + kHalf + kBlockM), t1 = __ldcg(p + kHalf + 2 * kBlockM);
-            v[u][0] = live ? m0 : -INFINITY; v[u][1] = live ? s_0 : 0.0f; v[u][2] = live ? t0 : -INFINITY;
-            v[u][3] = live ? m1 : -INFINITY; v[u][4] = live ? s_1 : 0.0f; v[u][5] = live ? t1 : -INFINITY;
+            f.marked = f.marked || (live && (s_0 < 0.0f || s_1 < 0.0f));
+            v[u][0] = live ? m0 : -INFINITY; v[u][1] = live ? fabsf(s_0) : 0.0f; v[u][2] = live ? t0 : -INFINITY;
+            v[u][3] = live ? m1 : -INFINITY; v[u][4] = live ? fabsf(s_1) : 0.0f; v[u][5] = live ? t1 : -INFINITY;
         }
 #pragma unroll
         for (int u = 0; u < kMergeBatch; ++u) {
@@ -74,11 +79,9 @@ __device__ __forceinline__ RowFold fold_row(const ScorePlan& plan, const float* 
     return f;
 }
 
-// log pi_target of the drafted token of `row`:  logit - (max + log2 sum) * ln 2.
-__device__ __forceinline__ float merged_logprob(const ScorePlan& plan, const float* __restrict__ workspace,
-                                                int64_t row, int32_t id, uint32_t* __restrict__ status) {
-    const RowFold f = fold_row(plan, workspace, row);
-    if (id < 0 || id >= plan.V) {
+// log pi_target of the drafted token from a row's fold:  logit - (max + log2 sum) * ln 2.
+__device__ __forceinline__ float fold_logprob(const RowFold& f, int32_t id, int32_t V, uint32_t* __restrict__ status) {
+    if (id < 0 || id >= V) {
         atomicOr(status, SPECS_DEV_TOKEN_RANGE);
         return __int_as_float(0x7fc00000);                  // no such vocabulary entry: NaN
     }
@@ -86,14 +89,88 @@ __device__ __forceinline__ float merged_logprob(const ScorePlan& plan, const flo
     return (float)((double)f.logit - lse);
 }
 
-// One row's fold as it stands, for a holder of one shard of the vocabulary: partials[row] =
-// (max in base-2 units, sum of 2^(x - max), drafted id's logit or -inf, 0).
-__global__ void __launch_bounds__(128)
-row_partials_kernel(const ScorePlan plan, const float* __restrict__ workspace, float4* __restrict__ partials) {
+// What the merge needs to collect the marked rows of an adaptive plan (ctl == NULL otherwise).
+struct CollectArgs {
+    FixCtl* ctl;
+    int32_t* list;                // [cap_rows]
+    uint8_t* compact;             // [cap_rows, row_bytes]
+    float* compact_scale;         // [cap_rows], 8-bit operands only
+    const uint8_t* hidden;        // [rows, row_bytes]
+    const float* hidden_scale;    // [rows] or NULL
+    int32_t row_bytes;            // a multiple of 16
+    int32_t cap_rows;
+};
+constexpr int kMergeThreads = 128;
+
+// One thread per row: fold the first pass's splits and write the row's log-probability (or, for a holder
+// of one vocabulary shard, its partials: max in base-2 units, sum of 2^(x - max), drafted id's logit or
+// -inf, 0).  A marked row also takes the next place in the list of rows to re-score; then the CTA's
+// threads together copy the hidden states of the CTA's marked rows into the compact buffer.  Rows beyond
+// the buffer's capacity are only counted: the second pass then works on all rows in place.
+__global__ void __launch_bounds__(kMergeThreads)
+merge_splits_kernel(const ScorePlan plan, const float* __restrict__ workspace,
+                    const int32_t* __restrict__ token_ids, float* __restrict__ tok_logprob,
+                    float4* __restrict__ partials, const CollectArgs col, uint32_t* __restrict__ status) {
+    __shared__ int32_t marked_row[kMergeThreads], marked_at[kMergeThreads];
+    __shared__ int marked_n;
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // the scoring kernel's results
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (threadIdx.x == 0) marked_n = 0;
+    __syncthreads();
     const int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (row >= plan.rows) return;
-    const RowFold f = fold_row(plan, workspace, row);
-    partials[row] = make_float4(f.max2, (float)f.sum2, f.logit, 0.0f);
+    if (row < plan.rows) {
+        const RowFold f = fold_row(plan, workspace, row);
+        if (partials) partials[row] = make_float4(f.max2, (float)f.sum2, f.logit, 0.0f);
+        else          tok_logprob[row] = fold_logprob(f, token_ids[row], plan.V, status);
+        if (f.marked && col.ctl != nullptr) {
+            const uint32_t at = atomicAdd(&col.ctl->count, 1u);
+            if (at < (uint32_t)col.cap_rows) {
+                col.list[at] = (int32_t)row;
+                if (col.compact_scale) col.compact_scale[at] = col.hidden_scale[row];
+                const int k = atomicAdd(&marked_n, 1);
+                marked_row[k] = (int32_t)row;
+                marked_at[k] = (int32_t)at;
+            }
+        }
+    }
+    if (col.ctl == nullptr) return;
+    __syncthreads();
+    const int n = marked_n;
+    const int vecs = col.row_bytes / 16;
+    for (int k = 0; k < n; ++k) {
+        const uint4* src = reinterpret_cast<const uint4*>(col.hidden + (size_t)marked_row[k] * col.row_bytes);
+        uint4* dst = reinterpret_cast<uint4*>(col.compact + (size_t)marked_at[k] * col.row_bytes);
+        for (int v = threadIdx.x; v < vecs; v += kMergeThreads) dst[v] = __ldg(src + v);
+    }
+}
+
+// How the second pass ran, from the number of marked rows: not at all, over the gathered rows, or over
+// every row in place.  `*plan2` is then the plan its slots are laid out by.
+__device__ __forceinline__ int second_pass_rows(const ScorePlan& plan, const FixView& fix, ScorePlan* plan2,
+                                                bool* compact) {
+    if (fix.ctl == nullptr) return 0;
+    const uint32_t n = *reinterpret_cast<const volatile uint32_t*>(&fix.ctl->count);
+    if (n == 0u) return 0;
+    *compact = n <= (uint32_t)fix.cap_rows;
+    *plan2 = *compact ? make_compact_plan(plan, (int64_t)n) : make_inplace_fix_plan(plan);
+    return *compact ? (int)n : (int)plan.rows;
+}
+
+// Results of the second pass over those of the re-scored rows: one thread per re-scored row.
+__global__ void __launch_bounds__(kMergeThreads)
+fix_merge_kernel(const ScorePlan plan, const FixView fix, const int32_t* __restrict__ token_ids,
+                 float* __restrict__ tok_logprob, float4* __restrict__ partials, uint32_t* __restrict__ status) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    ScorePlan plan2;
+    bool compact = false;
+    const int n = second_pass_rows(plan, fix, &plan2, &compact);
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int64_t row = compact ? (int64_t)fix.list[i] : i;
+    const RowFold f = fold_row(plan2, fix.slots, i);
+    if (partials) partials[row] = make_float4(f.max2, (float)f.sum2, f.logit, 0.0f);
+    else          tok_logprob[row] = fold_logprob(f, token_ids[row], plan.V, status);
 }
 
 // The same fold over the shards' partials [shards, rows]: log pi_target of the drafted id.
@@ -121,16 +198,6 @@ merge_partials_kernel(const float4* __restrict__ partials, int32_t shards, int64
         return;
     }
     tok_logprob[row] = (float)((double)logit - ((double)m + log2(sum)) * kLn2);
-}
-
-__global__ void __launch_bounds__(128)
-merge_splits_kernel(const ScorePlan plan, const float* __restrict__ workspace,
-                    const int32_t* __restrict__ token_ids, float* __restrict__ tok_logprob,
-                    uint32_t* __restrict__ status) {
-    // one thread per row; consecutive lanes read consecutive floats of a slot
-    const int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (row >= plan.rows) return;
-    tok_logprob[row] = merged_logprob(plan, workspace, row, token_ids[row], status);
 }
 
 // ------------------------------------------------------------------------------------ block sums
@@ -295,10 +362,10 @@ __global__ void select_kernel(const double* __restrict__ lp_t, const double* __r
 }
 
 // ------------------------------------------------------------------------------------ fused finish
-// Everything after the LM-head pass for one problem per CTA: merge the vocabulary splits of the
-// problem's rows, sum target and generator log-probabilities per drafted block, then SubSample and
-// the switch test on those sums.  The three phases are separated by CTA barriers; the block sums
-// travel through the output arrays blk_lp / gen_lp (double).  One launch instead of four.
+// Everything after the merge for one problem per CTA: where a second scoring pass ran, its results go over
+// those of the problem's re-scored rows first; then target and generator log-probabilities are summed per
+// drafted block, then SubSample and the switch test on those sums.  The phases are separated by CTA
+// barriers; the block sums travel through the output arrays blk_lp / gen_lp (double).
 constexpr int kFinishThreads = 1024;
 
 // Ids of the selected block of problem p into row p of chosen_ids [P, stride] (-1 beyond the block's
@@ -328,18 +395,37 @@ __global__ void gather_chosen_kernel(const int32_t* __restrict__ token_ids, cons
                         threadIdx.x, blockDim.x);
 }
 
-// With workspace_g the generator's per-token log-probabilities are not an input: they are merged from
-// a second scoring pass (the generator's own LM head on the same drafted ids) and written to gen_tok.
+// Second-pass results of the rows [row_a, row_b) into `tok`.
+__device__ __forceinline__ void apply_second_pass(const ScorePlan& plan, const FixView& fix, int64_t row_a,
+                                                  int64_t row_b, const int32_t* __restrict__ token_ids, float* tok,
+                                                  uint32_t* __restrict__ status, int tid, int nthreads) {
+    ScorePlan plan2;
+    bool compact = false;
+    const int n = second_pass_rows(plan, fix, &plan2, &compact);
+    if (n == 0) return;
+    if (compact) {
+        for (int i = tid; i < n; i += nthreads) {
+            const int64_t row = fix.list[i];
+            if (row >= row_a && row < row_b)
+                tok[row] = fold_logprob(fold_row(plan2, fix.slots, i), token_ids[row], plan.V, status);
+        }
+    } else {
+        for (int64_t row = row_a + tid; row < row_b; row += nthreads)
+            tok[row] = fold_logprob(fold_row(plan2, fix.slots, row), token_ids[row], plan.V, status);
+    }
+}
+
+// tok_logprob (and, with two scoring passes, gen_tok) hold the merged first-pass results; gen_tok may also
+// be the caller's own array of generator log-probabilities (fix_g.ctl == NULL then), or NULL.
 __global__ void __launch_bounds__(kFinishThreads)
-finish_step_kernel(const ScorePlan plan, const float* __restrict__ workspace, const ScorePlan plan_g,
-                   const float* __restrict__ workspace_g, const int32_t* __restrict__ token_ids,
-                   const int64_t* __restrict__ block_offsets, const int32_t* __restrict__ cand_offsets,
-                   float* gen_tok, const float* __restrict__ reward, const float* __restrict__ uniforms, float beta,
-                   float tau, float* __restrict__ tok_logprob, double* blk_lp, double* gen_lp,
-                   float* __restrict__ weights, int32_t* chosen, uint8_t* __restrict__ accept,
+finish_step_kernel(const ScorePlan plan, const FixView fix_t, const ScorePlan plan_g, const FixView fix_g,
+                   const int32_t* __restrict__ token_ids, const int64_t* __restrict__ block_offsets,
+                   const int32_t* __restrict__ cand_offsets, float* gen_tok, const float* __restrict__ reward,
+                   const float* __restrict__ uniforms, float beta, float tau, float* tok_logprob, double* blk_lp,
+                   double* gen_lp, float* __restrict__ weights, int32_t* chosen, uint8_t* __restrict__ accept,
                    int32_t* __restrict__ chosen_ids, int32_t* __restrict__ chosen_len, int32_t chosen_stride,
                    uint32_t* __restrict__ status) {
-    // Launched with programmatic stream serialisation: wait here for the scoring kernel's results.
+    // Launched with programmatic stream serialisation: wait here for the kernels before it.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // let the next kernel of the stream (the next step's scoring kernel) begin its prologue
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -348,12 +434,11 @@ finish_step_kernel(const ScorePlan plan, const float* __restrict__ workspace, co
     const int a = cand_offsets[p], b = cand_offsets[p + 1];
     if (b > a) {
         const int64_t row_a = block_offsets[a], row_b = block_offsets[b];   // the problem's rows are contiguous
-        for (int64_t row = row_a + threadIdx.x; row < row_b; row += kFinishThreads) {
-            const int32_t id = token_ids[row];
-            tok_logprob[row] = merged_logprob(plan, workspace, row, id, status);
-            if (workspace_g) gen_tok[row] = merged_logprob(plan_g, workspace_g, row, id, status);
+        if (fix_t.ctl != nullptr || fix_g.ctl != nullptr) {
+            apply_second_pass(plan, fix_t, row_a, row_b, token_ids, tok_logprob, status, threadIdx.x, kFinishThreads);
+            apply_second_pass(plan_g, fix_g, row_a, row_b, token_ids, gen_tok, status, threadIdx.x, kFinishThreads);
+            __syncthreads();
         }
-        __syncthreads();
         for (int i = a + warp; i < b; i += kFinishThreads / 32) {
             const int64_t t0 = block_offsets[i], t1 = block_offsets[i + 1];
             double lp = 0.0, lq = 0.0;
@@ -439,36 +524,66 @@ inline unsigned warps_grid(int64_t warps, int threads) {
 
 }  // namespace
 
-int launch_merge(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, const int32_t* token_ids,
-                 float* tok_logprob, cudaStream_t stream) {
-    if (plan.rows == 0) return SPECS_OK;
-    const unsigned blocks = (unsigned)((plan.rows + 127) / 128);
-    merge_splits_kernel<<<blocks, 128, 0, stream>>>(plan, workspace, token_ids, tok_logprob, ctx->d_status);
-    return cuda_status(cudaGetLastError());
-}
-
-int launch_finish_step(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, const ScorePlan* plan_g,
-                       const float* workspace_g, const int32_t* token_ids, const int64_t* block_offsets,
-                       const int32_t* cand_offsets, int32_t P, float* gen_tok, const float* reward,
-                       const float* uniforms, float beta, float tau, float* tok_logprob, double* blk_lp, double* gen_lp,
-                       float* weights, int32_t* chosen, uint8_t* accept, int32_t* chosen_ids, int32_t* chosen_len,
-                       int32_t chosen_stride, cudaStream_t stream) {
-    if (P == 0) return SPECS_OK;
+namespace {
+// every kernel of a step is launched with programmatic stream serialisation and waits for its predecessor itself
+template <typename... KArgs, typename... Args>
+int launch_chained(void (*kernel)(KArgs...), unsigned blocks, unsigned threads, cudaStream_t stream, Args... args) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)P, 1, 1);
-    cfg.blockDim = dim3(kFinishThreads, 1, 1);
+    cfg.gridDim = dim3(blocks, 1, 1);
+    cfg.blockDim = dim3(threads, 1, 1);
     cfg.stream = stream;
-    // the launch is set up while the scoring kernel still runs; the kernel itself waits for it
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
+    return cuda_status(cudaLaunchKernelEx(&cfg, kernel, args...));
+}
+}  // namespace
+
+int launch_merge(specs_ctx* ctx, const ScorePlan& plan, void* workspace, const int32_t* token_ids,
+                 float* tok_logprob, float* partials, const void* hidden, const float* hidden_scale,
+                 cudaStream_t stream) {
+    if (plan.rows == 0) return SPECS_OK;
+    CollectArgs col = {};
+    if (plan.adaptive) {
+        const WsLayout lay = plan_layout(plan);
+        uint8_t* ws = static_cast<uint8_t*>(workspace);
+        col.ctl = reinterpret_cast<FixCtl*>(ws + lay.ctl);
+        col.list = reinterpret_cast<int32_t*>(ws + lay.list);
+        col.compact = ws + lay.compact;
+        col.compact_scale = plan.elem_bytes == 1 ? reinterpret_cast<float*>(ws + lay.compact_scale) : nullptr;
+        col.hidden = static_cast<const uint8_t*>(hidden);
+        col.hidden_scale = hidden_scale;
+        col.row_bytes = plan.d * plan.elem_bytes;
+        col.cap_rows = lay.cap_rows;
+    }
+    const unsigned blocks = (unsigned)((plan.rows + kMergeThreads - 1) / kMergeThreads);
+    return launch_chained(merge_splits_kernel, blocks, kMergeThreads, stream, plan,
+                          static_cast<const float*>(workspace), token_ids, tok_logprob,
+                          reinterpret_cast<float4*>(partials), col, ctx->d_status);
+}
+
+int launch_fix_merge(specs_ctx* ctx, const ScorePlan& plan, const void* workspace, const int32_t* token_ids,
+                     float* tok_logprob, float* partials, cudaStream_t stream) {
+    if (plan.rows == 0 || !plan.adaptive) return SPECS_OK;
+    const unsigned blocks = (unsigned)((plan.rows + kMergeThreads - 1) / kMergeThreads);
+    return launch_chained(fix_merge_kernel, blocks, kMergeThreads, stream, plan, fix_view(plan, workspace), token_ids,
+                          tok_logprob, reinterpret_cast<float4*>(partials), ctx->d_status);
+}
+
+int launch_finish_step(specs_ctx* ctx, const ScorePlan& plan, const FixView& fix_t, const ScorePlan* plan_g,
+                       const FixView& fix_g, const int32_t* token_ids, const int64_t* block_offsets,
+                       const int32_t* cand_offsets, int32_t P, float* gen_tok, const float* reward,
+                       const float* uniforms, float beta, float tau, float* tok_logprob, double* blk_lp, double* gen_lp,
+                       float* weights, int32_t* chosen, uint8_t* accept, int32_t* chosen_ids, int32_t* chosen_len,
+                       int32_t chosen_stride, cudaStream_t stream) {
+    if (P == 0) return SPECS_OK;
     const ScorePlan second = plan_g ? *plan_g : plan;
-    return cuda_status(cudaLaunchKernelEx(&cfg, finish_step_kernel, plan, workspace, second, workspace_g, token_ids,
-                                          block_offsets, cand_offsets, gen_tok, reward, uniforms, beta, tau,
-                                          tok_logprob, blk_lp, gen_lp, weights, chosen, accept, chosen_ids, chosen_len,
-                                          chosen_stride, ctx->d_status));
+    return launch_chained(finish_step_kernel, (unsigned)P, kFinishThreads, stream, plan, fix_t, second, fix_g,
+                          token_ids, block_offsets, cand_offsets, gen_tok, reward, uniforms, beta, tau, tok_logprob,
+                          blk_lp, gen_lp, weights, chosen, accept, chosen_ids, chosen_len, chosen_stride,
+                          ctx->d_status);
 }
 
 int launch_gather_chosen(const int32_t* token_ids, const int64_t* block_offsets, const int32_t* cand_offsets,
@@ -477,15 +592,6 @@ int launch_gather_chosen(const int32_t* token_ids, const int64_t* block_offsets,
     if (P == 0) return SPECS_OK;
     gather_chosen_kernel<<<(unsigned)P, 128, 0, stream>>>(token_ids, block_offsets, cand_offsets, chosen, chosen_ids,
                                                           chosen_len, stride);
-    return cuda_status(cudaGetLastError());
-}
-
-int launch_row_partials(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, float* partials,
-                        cudaStream_t stream) {
-    (void)ctx;
-    if (plan.rows == 0) return SPECS_OK;
-    row_partials_kernel<<<(unsigned)((plan.rows + 127) / 128), 128, 0, stream>>>(plan, workspace,
-                                                                               reinterpret_cast<float4*>(partials));
     return cuda_status(cudaGetLastError());
 }
 

@@ -69,9 +69,72 @@ ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, i
                           int32_t cta_group = kCtaGroupAuto, int32_t chunk_kblocks = kDefaultChunkKBlocks,
                           bool adaptive = true, int32_t elem_bytes = 2);
 size_t plan_workspace_bytes(const ScorePlan& p);
-// The workspace: triple slots [waves x grid], then one 64-bit progress word per unit.
 __host__ __device__ inline size_t plan_slot_bytes(const ScorePlan& p) {
     return (size_t)(p.waves > 0 ? p.waves : 1) * (size_t)p.grid * kTripleFloats * sizeof(float);
+}
+
+// ---- second pass over the rows whose logits outgrew their tile's accumulation chunks --------------
+// With adaptive chunks the first pass marks every row in which a logit that matters (the row's
+// maximum or the drafted id's) lies beyond the magnitude its tile's chunks were sized for.  The merge
+// collects those rows (a count and a list), copies their hidden states into a compact buffer, and a
+// second launch of the scoring kernel re-scores them with the base chunks.  More marked rows than
+// the compact buffer holds: the second launch re-scores every row in place instead.
+struct FixCtl {
+    uint32_t count;        // rows marked by the merge (may exceed the compact capacity)
+    uint32_t pad[3];
+};
+
+// The workspace: triple slots [waves x grid], one 64-bit progress word per unit, and for adaptive
+// plans the control block, the list of marked rows, their gathered hidden states (and, for 8-bit
+// operands, row scales), and the slots + progress words of the second pass.
+struct WsLayout {
+    size_t progress;       // = plan_slot_bytes(plan)
+    size_t ctl, list, compact, compact_scale, fix_slots;   // 0 when the plan is not adaptive
+    size_t total;
+    int32_t cap_rows;      // rows the compact buffer holds (a multiple of the super tile)
+};
+inline WsLayout plan_layout(const ScorePlan& p) {
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    WsLayout L = {};
+    L.progress = plan_slot_bytes(p);
+    const size_t first = L.progress + (size_t)p.units * sizeof(uint64_t);
+    if (!p.adaptive) { L.total = first; return L; }
+    int cap_super = (p.super_tiles + 7) / 8;
+    if (cap_super > 32) cap_super = 32;
+    if (cap_super > p.units) cap_super = p.units;
+    if (cap_super < 1) cap_super = 1;
+    L.cap_rows = cap_super * kBlockM * p.cta_group;
+    size_t off = up(first);
+    L.ctl = off;            off += 256;
+    L.list = off;           off += up((size_t)L.cap_rows * sizeof(int32_t));
+    L.compact = off;        off += up((size_t)L.cap_rows * p.d * p.elem_bytes);
+    L.compact_scale = off;  off += p.elem_bytes == 1 ? up((size_t)L.cap_rows * sizeof(float)) : 0;
+    L.fix_slots = off;      off += up(first);
+    L.total = off;
+    return L;
+}
+
+// Plan of the second pass over `n` gathered rows (n <= cap_rows, so one wave): same tile shape and
+// vocabulary as `base`, every super tile live at once, the units shared out over vocabulary chunks,
+// base chunks throughout.
+__host__ __device__ inline ScorePlan make_compact_plan(const ScorePlan& base, int64_t n) {
+    ScorePlan p = base;
+    p.rows = n;
+    p.row_tiles = (int32_t)((n + kBlockM - 1) / kBlockM);
+    p.super_tiles = (p.row_tiles + p.cta_group - 1) / p.cta_group;
+    int s = p.super_tiles > 0 ? p.units / p.super_tiles : 1;
+    if (s > p.vocab_tiles) s = p.vocab_tiles;
+    if (s < 1) s = 1;
+    p.group_m = p.super_tiles; p.split_full = s; p.full_waves = p.super_tiles > 0 ? 1 : 0;
+    p.rem_m = 0; p.split_rem = 0; p.waves = p.full_waves;
+    p.adaptive = 0;
+    return p;
+}
+// The second pass over all rows in place: the first pass's geometry with the base chunks.
+__host__ __device__ inline ScorePlan make_inplace_fix_plan(const ScorePlan& base) {
+    ScorePlan p = base;
+    p.adaptive = 0;
+    return p;
 }
 
 // Work unit `unit` in wave `wave`: returns false when the unit idles in that wave.
@@ -93,7 +156,22 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-struct TimedLaunch { cudaEvent_t start, stop; };
+struct TimedLaunch { cudaEvent_t start, stop; bool second_pass; };
+
+// A tensor map the context has encoded before, found again by what it describes.
+struct CachedMap {
+    const void* base; uint64_t inner, outer; uint32_t box_inner, box_outer; int elem_bytes;
+    CUtensorMap map;
+};
+constexpr size_t kMapCacheSize = 16;
+
+// What the kernels after the first scoring pass need to know about the second one.
+struct FixView {
+    const FixCtl* ctl;        // NULL: the plan is not adaptive, there is no second pass
+    const int32_t* list;      // marked rows in the order of the compact buffer
+    const float* slots;       // triple slots of the second pass
+    int32_t cap_rows;
+};
 
 }  // namespace specs
 
@@ -112,6 +190,8 @@ struct specs_ctx {
     size_t arena_bytes = 0;
     void* h_stage = nullptr;               // pinned mirror of the arena's small-input and output blocks
     size_t stage_bytes = 0;
+    std::vector<specs::CachedMap> maps;    // tensor maps of recent operands (round robin)
+    size_t maps_next = 0;
     // optional per-launch timing of the tensor-core kernel
     bool timing = false;
     std::vector<specs::TimedLaunch> timed;
@@ -124,17 +204,32 @@ namespace specs {
 // CTA pairs of the pair kernel that the current device keeps resident at once (cached per
 // device; also opts both kernels in to their dynamic shared memory).  0 if pairs cannot launch.
 int query_pair_units(int device, int num_sms);
+// First pass: scores every row; `workspace` is laid out by plan_layout(plan).
 int launch_score_tcgen05(specs_ctx* ctx, const ScorePlan& plan, const void* hidden, const void* w_vocab,
-                         const int32_t* token_ids, float* workspace, cudaStream_t stream, int32_t id_offset = 0,
+                         const int32_t* token_ids, void* workspace, cudaStream_t stream, int32_t id_offset = 0,
                          const float* hidden_scale = nullptr, const float* w_scale = nullptr);
+// Second pass (adaptive plans only; a no-op launch when the merge marked no row): re-scores the marked
+// rows with the base chunks.  Must follow launch_merge on the same workspace.
+int launch_score_second_pass(specs_ctx* ctx, const ScorePlan& plan, const void* hidden, const void* w_vocab,
+                             const int32_t* token_ids, void* workspace, cudaStream_t stream, int32_t id_offset = 0,
+                             const float* hidden_scale = nullptr, const float* w_scale = nullptr);
+FixView fix_view(const ScorePlan& plan, const void* workspace);
 int launch_quantize_rows(const void* x_bf16, int64_t n, int32_t d, uint8_t* codes, float* scale, cudaStream_t stream);
 int launch_wait_expiry_probe(specs_ctx* ctx, unsigned long long limit_ns, cudaStream_t stream);
 int launch_score_simt(specs_ctx* ctx, const void* hidden, const void* w_vocab, const int32_t* token_ids,
                       int64_t rows, int32_t d, int32_t V, float* tok_logprob, cudaStream_t stream);
-int launch_merge(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, const int32_t* token_ids,
-                 float* tok_logprob, cudaStream_t stream);
-int launch_finish_step(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, const ScorePlan* plan_g,
-                       const float* workspace_g, const int32_t* token_ids, const int64_t* block_offsets,
+// Merge of the first pass's splits into tok_logprob (or, with `partials`, into per-row shard partials);
+// for adaptive plans it also collects the marked rows and gathers their hidden states.
+int launch_merge(specs_ctx* ctx, const ScorePlan& plan, void* workspace, const int32_t* token_ids,
+                 float* tok_logprob, float* partials, const void* hidden, const float* hidden_scale,
+                 cudaStream_t stream);
+// Results of the second pass written over those of the marked rows.
+int launch_fix_merge(specs_ctx* ctx, const ScorePlan& plan, const void* workspace, const int32_t* token_ids,
+                     float* tok_logprob, float* partials, cudaStream_t stream);
+// Block sums of both per-token arrays, SubSample, the switch test and the gather of the chosen block, one CTA
+// per problem.  fix_t / fix_g: second-pass results still to be written over tok_logprob / gen_tok first.
+int launch_finish_step(specs_ctx* ctx, const ScorePlan& plan, const FixView& fix_t, const ScorePlan* plan_g,
+                       const FixView& fix_g, const int32_t* token_ids, const int64_t* block_offsets,
                        const int32_t* cand_offsets, int32_t P, float* gen_tok, const float* reward,
                        const float* uniforms, float beta, float tau, float* tok_logprob, double* blk_lp, double* gen_lp,
                        float* weights, int32_t* chosen, uint8_t* accept, int32_t* chosen_ids, int32_t* chosen_len,
@@ -142,8 +237,6 @@ int launch_finish_step(specs_ctx* ctx, const ScorePlan& plan, const float* works
 int launch_gather_chosen(const int32_t* token_ids, const int64_t* block_offsets, const int32_t* cand_offsets,
                          const int32_t* chosen, int32_t P, int32_t* chosen_ids, int32_t* chosen_len, int32_t stride,
                          cudaStream_t stream);
-int launch_row_partials(specs_ctx* ctx, const ScorePlan& plan, const float* workspace, float* partials,
-                        cudaStream_t stream);
 int launch_merge_partials(specs_ctx* ctx, const float* partials, int32_t shards, int64_t rows, const int32_t* token_ids,
                           int32_t V, float* tok_logprob, cudaStream_t stream);
 int launch_block_sums(const float* per_token, const int64_t* block_offsets, int32_t B,

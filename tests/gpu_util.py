@@ -63,12 +63,28 @@ BLK_RTOL = 1e-2
 MARGIN = 1e-3
 
 
+# The end-to-end pick is compared where the oracle's margin exceeds MARGIN plus a slack for the rounding the
+# two compared block log-probs carry on the GPU side.  That slack is bounded: a block sum may be off by an
+# eighth of the per-token tolerance per token (the error of a token is mostly a bias of one sign, so it adds
+# up along a block), and never less than MAX_PICK_SLACK is allowed.
+MAX_PICK_SLACK = 1e-2
+
+
+def pick_slack(got_blk, want_blk, max_block_len=0):
+    """Slack on the pick margin of one problem: twice the largest block log-prob error observed in it."""
+    slack = 2.0 * float(np.abs(np.asarray(got_blk) - np.asarray(want_blk)).max(initial=0.0))
+    bound = max(MAX_PICK_SLACK, 2.0 * max_block_len * TOK_ATOL / 8.0)
+    assert slack <= bound, f"block log-prob error widens the pick exemption to {slack:.3e} (bound {bound:.3e})"
+    return slack
+
+
 def assert_step_matches(got, want, cand_offsets, block_offsets, lp_slack_per_token=0.0):
     """Compare a full step's outputs with the oracle's.
 
     The pick is compared where the oracle's margin exceeds MARGIN plus the worst-case shift the
-    block log-prob error can cause in a perturbed-score difference (two blocks, every token off by
-    the per-token tolerance actually observed).
+    block log-prob error can cause in a perturbed-score difference (two blocks, each off by the
+    largest block error observed in the problem); that slack is bounded by MAX_PICK_SLACK, and the
+    number of problems it exempted (beyond those under the plain MARGIN rule) is returned.
     """
     tok_err = np.abs(got["tok_logprob"] - want["tok_logprob"])
     assert np.all(np.isfinite(got["tok_logprob"])), "non-finite token log-prob"
@@ -80,18 +96,21 @@ def assert_step_matches(got, want, cand_offsets, block_offsets, lp_slack_per_tok
         assert rel[nz].max(initial=0.0) <= BLK_RTOL, f"{key} relative error {rel[nz].max():.3e}"
     lens = np.diff(block_offsets)
     P = len(cand_offsets) - 1
-    exact = 0
+    exact, by_slack, max_slack = 0, 0, 0.0
     for p in range(P):
         a, b = cand_offsets[p], cand_offsets[p + 1]
         if b <= a:
             assert got["chosen"][p] == -1
             continue
-        blk_err = np.abs(got["blk_logprob_f64"][a:b] - want["blk_logprob"][a:b])
-        slack = 2.0 * blk_err.max()
+        slack = pick_slack(got["blk_logprob_f64"][a:b], want["blk_logprob"][a:b], int(lens[a:b].max()))
+        max_slack = max(max_slack, slack)
         if want["margin"][p] > MARGIN + slack:
             assert got["chosen"][p] == want["chosen"][p], (p, want["margin"][p], slack)
             exact += 1
         else:
             assert 0 <= got["chosen"][p] < b - a
+            if want["margin"][p] > MARGIN:
+                by_slack += 1
     assert np.array_equal(got["accept"], want["accept"])
-    return {"tok_max_err": float(tok_err.max()), "picks_checked_exactly": exact, "problems": P}
+    return {"tok_max_err": float(tok_err.max()), "picks_checked_exactly": exact, "problems": P,
+            "picks_exempted_by_slack": by_slack, "max_pick_slack": max_slack}

@@ -13,7 +13,7 @@ import torch
 from oracle import specs_oracle as O
 from paper_2506_15733_b200 import binding
 from paper_2506_15733_b200 import inputs as I
-from tests.gpu_util import BLK_RTOL, MARGIN, TOK_ATOL, DeviceStep
+from tests.gpu_util import BLK_RTOL, MARGIN, TOK_ATOL, DeviceStep, pick_slack
 
 pytestmark = pytest.mark.gpu
 
@@ -99,7 +99,7 @@ def test_step7b_all_rows_all_betas(ctx, engine):
         # end to end: oracle block log-probs vs GPU block log-probs
         S = O.scores(LP, LQ, x.reward, beta)
         want_c, margin = O.gumbel_pick(S, x.uniforms, x.cand_offsets)
-        slack = 2 * np.abs(g["blk_logprob_f64"] - LP).max()
+        slack = pick_slack(g["blk_logprob_f64"], LP, 64)
         if margin[0] > MARGIN + slack:
             assert g["chosen"][0] == want_c[0]
         assert np.abs(g["weights"] - O.weights(S, x.cand_offsets)).max() < 5e-3 + 2 * slack
@@ -124,7 +124,7 @@ def test_batched_ragged_step(ctx):
     LP0 = np.array([sum(by_row[t] for t in range(x.block_offsets[b], x.block_offsets[b + 1])) for b in range(8)])
     S0 = O.scores(LP0, LQ[:8], x.reward[:8], 2.0)
     c0, m0 = O.gumbel_pick(S0, x.uniforms[:8], np.array([0, 8]))
-    slack = 2 * np.abs(got["blk_logprob_f64"][:8] - LP0).max()
+    slack = pick_slack(got["blk_logprob_f64"][:8], LP0, 128)
     if m0[0] > MARGIN + slack:
         assert got["chosen"][0] == c0[0]
     # selection logic on all 32 problems, and the threshold sweep
@@ -134,13 +134,32 @@ def test_batched_ragged_step(ctx):
         assert check_selection_logic(x, s.results(), 2.0, tau, LQ) >= 24
 
 
+def check_problem_end_to_end(x, got_chosen, got_blk, p, LP, LQ, beta):
+    """Oracle scores, pick and margin of one problem whose blocks the oracle scored in full."""
+    a, b = int(x.cand_offsets[p]), int(x.cand_offsets[p + 1])
+    S = O.scores(LP, LQ, x.reward[a:b], beta)
+    want_c, margin = O.gumbel_pick(S, x.uniforms[a:b], np.array([0, b - a]))
+    slack = pick_slack(got_blk[a:b], LP, int(np.diff(x.block_offsets)[a:b].max()))
+    if margin[0] > MARGIN + slack:
+        assert got_chosen[p] == want_c[0], (p, margin[0], slack)
+        return 1
+    return 0
+
+
 @pytest.mark.parametrize("token_dist", ["zipf", "zipf_perm"])
 def test_dual_scoring_draft_then_target(ctx, token_dist):
     # the same 65536 drafted tokens scored with a 1.5B-draft-shaped head and a 7B-target-shaped head;
-    # the draft pass supplies the generator's block log-probs (Eq. 1's denominator)
+    # the draft pass supplies the generator's block log-probs (Eq. 1's denominator).  For the plain Zipf
+    # ids the oracle scores one whole problem (32 blocks of 256 tokens) per pass, which also allows the
+    # end-to-end pick of that problem; for the permuted ids three blocks and 128 single rows.
     rng = np.random.Generator(np.random.Philox(key=[7003, 1]))
-    blocks = sorted(rng.choice(256, size=3, replace=False).tolist())
-    blk = {}
+    if token_dist == "zipf":
+        problem = int(rng.integers(8))
+        blocks = list(range(32 * problem, 32 * problem + 32))
+    else:
+        problem = None
+        blocks = sorted(rng.choice(256, size=3, replace=False).tolist())
+    blk, oracle_blk = {}, {}
     for name in ("dual_draft", "dual_target"):
         cfg = I.scaled(I.CONFIGS[name], token_dist=token_dist)
         x = I.make_step_inputs(cfg)
@@ -151,7 +170,12 @@ def test_dual_scoring_draft_then_target(ctx, token_dist):
         w64 = O.bf16_bits_to_f64(x.w_vocab)
         rows_idx = np.unique(np.concatenate([rows_of_blocks(x, blocks), rng.choice(x.rows, 128, replace=False)]))
         want_tok, err = check_sampled_rows(x, got["tok_logprob"], rows_idx, w64)
-        check_block_sums(x, got, blocks, dict(zip(rows_idx.tolist(), want_tok.tolist())))
+        by_row = dict(zip(rows_idx.tolist(), want_tok.tolist()))
+        check_block_sums(x, got, blocks, by_row)
+        oracle_blk[name] = np.array([O.block_sums(np.array([by_row[t] for t in range(x.block_offsets[b],
+                                                                                      x.block_offsets[b + 1])]),
+                                                  np.array([0, x.block_offsets[b + 1] - x.block_offsets[b]]))[0]
+                                     for b in blocks])
         blk[name] = s.blk_lp64.clone()
         keep = s
         del w64
@@ -162,6 +186,17 @@ def test_dual_scoring_draft_then_target(ctx, token_dist):
     g = keep.results()
     g["blk_logprob_f64"] = blk["dual_target"].cpu().numpy()
     assert check_selection_logic(x, g, 1.0, 0.7, blk["dual_draft"].cpu().numpy()) >= 6
+    if problem is not None:
+        # end to end on the whole problem: both block log-probs from the oracle; the slack covers the
+        # rounding of the GPU's target AND draft block sums
+        a = 32 * problem
+        gpu_ratio = g["blk_logprob_f64"] - blk["dual_draft"].cpu().numpy()
+        want_ratio = oracle_blk["dual_target"] - oracle_blk["dual_draft"]
+        S = O.scores(oracle_blk["dual_target"], oracle_blk["dual_draft"], x.reward[a:a + 32], 1.0)
+        want_c, margin = O.gumbel_pick(S, x.uniforms[a:a + 32], np.array([0, 32]))
+        slack = pick_slack(gpu_ratio[a:a + 32], want_ratio, 2 * 256)     # two block sums per candidate
+        if margin[0] > MARGIN + slack:
+            assert g["chosen"][problem] == want_c[0]
 
 
 def test_dual_head_step_at_full_size(ctx):
@@ -216,21 +251,34 @@ def test_stress_heavy_tailed_logits(ctx):
     x = I.make_step_inputs(cfg)
     s = DeviceStep(ctx, x)
     got = s.step(cfg.betas[0], 0.7)
+    # the outlier rows went through the second scoring pass (reported, not an error)
+    assert ctx.device_status() == binding.DEV_ACCUM_RANGE
     w64 = O.bf16_bits_to_f64(x.w_vocab)
     rng = np.random.Generator(np.random.Philox(key=[7004, 1]))
-    # blocks that contain outlier rows (shortest three of them), 160 outlier rows, 64 ordinary rows
+    # one whole problem chosen by seed (64 blocks), the eight blocks of the other problems that hold the
+    # most outlier rows, 160 more outlier rows and 64 more ordinary rows
+    problem = int(rng.integers(cfg.problems))
+    a, b = int(x.cand_offsets[problem]), int(x.cand_offsets[problem + 1])
+    assert b - a == 64
     blk_of_row = np.searchsorted(x.block_offsets, x.outlier_rows, side="right") - 1
-    cand_blocks = np.unique(blk_of_row)
-    lens = np.diff(x.block_offsets)[cand_blocks]
-    blocks = cand_blocks[np.argsort(lens)[:3]].tolist()
+    per_block = np.bincount(blk_of_row, minlength=x.blocks)
+    per_block[a:b] = -1
+    heavy = np.argsort(-per_block, kind="stable")[:8].tolist()
+    assert all(per_block[h] >= 1 for h in heavy)
+    blocks = list(range(a, b)) + sorted(heavy)
     rows_idx = np.unique(np.concatenate([rows_of_blocks(x, blocks),
                                          rng.choice(x.outlier_rows, 160, replace=False),
                                          rng.choice(x.rows, 64, replace=False)]))
+    assert np.isin(x.outlier_rows, rows_idx).sum() >= 160
     want_tok, err = check_sampled_rows(x, got["tok_logprob"], rows_idx, w64)
     assert np.abs(want_tok).max() > 100                       # the sample really holds heavy-tailed rows
-    check_block_sums(x, got, blocks, dict(zip(rows_idx.tolist(), want_tok.tolist())))
+    by_row = dict(zip(rows_idx.tolist(), want_tok.tolist()))
+    check_block_sums(x, got, blocks, by_row)
     LQ = O.block_sums(x.draft_tok_logprob, x.block_offsets)
+    LP = np.array([sum(by_row[t] for t in range(x.block_offsets[i], x.block_offsets[i + 1])) for i in range(a, b)])
     for beta in cfg.betas:
         s.select(beta, 0.7)
         torch.cuda.synchronize()
-        check_selection_logic(x, s.results(), beta, 0.7, LQ)
+        g = s.results()
+        check_selection_logic(x, g, beta, 0.7, LQ)
+        check_problem_end_to_end(x, g["chosen"], g["blk_logprob_f64"], problem, LP, LQ[a:b], beta)

@@ -415,29 +415,97 @@ def test_adaptive_chunks_keep_the_tolerance_across_logit_magnitudes(ctx, sigma_z
     assert np.abs(got[binding.ACCUM_ADAPTIVE] - got[512]).max() <= TOK_ATOL / 4
 
 
-def test_adaptive_chunks_flag_logits_beyond_the_sampled_magnitude(ctx):
-    # vocabulary entries from the second tile on are 128 times larger than the first tile's: the chunk
-    # length chosen from the first tile is too long for them, which the advisory status bit reports
+def _scale_rows_by_128(bits, rows):
+    """Exact multiplication by 128 of the given rows of a bf16 bit array (exponent + 7), zeros left alone."""
+    out = bits.copy()
+    sel = out[rows]
+    nz = (sel & 0x7f80) != 0
+    sel[nz] += np.uint16(7 << 7)
+    out[rows] = sel
+    return out
+
+
+def _last_tiles_of_runs(ctx, rows, d, V):
+    """Vocabulary tiles (of 256 entries) that end some work unit's run in the plan for these sizes."""
+    p = binding.score_plan(rows, d, V, ctx.sm_count())
+    ends = set()
+    for c in range(p["grid"]):
+        mt, nb, ne = binding.score_plan_unit(rows, d, V, ctx.sm_count(), 0, c)
+        if mt >= 0 and ne - nb >= 3:
+            ends.add(ne - 1)
+    return sorted(ends)
+
+
+@pytest.mark.parametrize("case", ["from_second_tile", "last_tile_of_each_run", "one_row", "more_rows_than_gathered"])
+def test_adaptive_chunks_rescore_rows_beyond_the_sampled_magnitude(ctx, case):
+    # Logits far larger than what the first vocabulary tile of a run showed: the chunk length chosen from
+    # that tile is too long for them.  Such rows are marked, re-scored with the base chunks in a second
+    # pass, and the per-token tolerance holds wherever in the vocabulary the large logits sit.
     d, V = 5120, 60000
-    cfg = small_config("adapt_surprise", (64, 64), 1, 4, d, V, seed=5300, w_sigma=1.0 / math.sqrt(d))
+    blocks = 12 if case == "more_rows_than_gathered" else 4
+    cfg = small_config("adapt_surprise", (64, 64), 1, blocks, d, V, seed=5300, w_sigma=1.0 / math.sqrt(d))
     x = I.make_step_inputs(cfg)
-    w = x.w_vocab.copy()
-    big = w[256:]
-    nz = (big & 0x7f80) != 0
-    big[nz] += np.uint16(7 << 7)                             # exponent + 7: exact multiplication by 128
-    x.w_vocab = w
+    if case in ("from_second_tile", "more_rows_than_gathered"):
+        x.w_vocab = _scale_rows_by_128(x.w_vocab, np.arange(256, V))
+    elif case == "last_tile_of_each_run":
+        tiles = _last_tiles_of_runs(ctx, x.rows, d, V)
+        assert tiles
+        x.w_vocab = _scale_rows_by_128(x.w_vocab, np.concatenate([np.arange(256 * t, min(256 * t + 256, V))
+                                                                  for t in tiles]))
+    else:
+        x.hidden = _scale_rows_by_128(x.hidden, np.array([37]))
     want = O.token_logprobs(x.hidden, x.w_vocab, x.token_ids)
+    assert np.abs(want).max() > 50                           # the case really holds large logits
     got = _score_only(ctx, x)
     assert np.all(np.isfinite(got))
-    assert np.abs(got - want).max() <= 2e-2                  # still close: the bias is a few 1e-3 at most
+    assert np.abs(got - want).max() <= TOK_ATOL
+    assert ctx.device_status() == binding.DEV_ACCUM_RANGE    # reported: some rows went through the second pass
+    # the fused step takes the second pass's results in its finish kernel: same bits
+    f = DeviceStep(ctx, x)
+    ctx.specs_beam_step(f.hidden, f.w_vocab, f.token_ids, f.block_offsets, f.cand_offsets, f.draft, f.reward,
+                        f.uniforms, 1.0, 0.7, f.tok_lp, f.blk_lp64, f.gen_blk64, f.weights, f.chosen, f.accept,
+                        f.workspace)
+    torch.cuda.synchronize()
+    assert np.array_equal(f.tok_lp.cpu().numpy(), got)
+    assert np.allclose(f.blk_lp64.cpu().numpy(), O.block_sums(got, x.block_offsets), rtol=1e-12)
     assert ctx.device_status() == binding.DEV_ACCUM_RANGE
+    # fixed short chunks need no second pass and agree
     ctx.set_accum_chunk(512)
     try:
-        got = _score_only(ctx, x)
+        fixed = _score_only(ctx, x)
     finally:
         ctx.set_accum_chunk(binding.ACCUM_ADAPTIVE)
     assert ctx.device_status() == 0
+    assert np.abs(fixed - want).max() <= TOK_ATOL
+    if case == "more_rows_than_gathered":
+        assert np.array_equal(fixed, got)                    # every row was re-scored in place, same plan, same chunks
+    elif case != "one_row":
+        # every row was re-scored with those chunks, under another cut of the vocabulary: rounding only
+        assert np.all(np.abs(fixed - got) <= 1e-4 * np.maximum(1.0, np.abs(want)))
+
+
+def test_one_large_row_does_not_shorten_its_tiles_chunks(ctx):
+    # 1 % of the rows 20 times larger (the stress recipe): only those rows are re-scored; the others
+    # keep the chunk length their own magnitude allows, and all meet the tolerance
+    d, V = 5120, 60000
+    cfg = small_config("adapt_outliers", (128, 128), 1, 6, d, V, seed=5301, w_sigma=6.0 / math.sqrt(d),
+                       outlier_frac=0.01, outlier_mult=20.0)
+    x = I.make_step_inputs(cfg)
+    assert 2 <= len(x.outlier_rows) <= 24
+    want = O.token_logprobs(x.hidden, x.w_vocab, x.token_ids)
+    got = _score_only(ctx, x)
+    assert ctx.device_status() == binding.DEV_ACCUM_RANGE
     assert np.abs(got - want).max() <= TOK_ATOL
+    ctx.set_accum_chunk(512)
+    try:
+        fixed = _score_only(ctx, x)
+    finally:
+        ctx.set_accum_chunk(binding.ACCUM_ADAPTIVE)
+    assert ctx.device_status() == 0
+    # the outlier rows were re-scored with the base chunks; the ordinary rows were not (different rounding)
+    o = x.outlier_rows
+    assert np.all(np.abs(got[o] - fixed[o]) <= 1e-4 * np.maximum(1.0, np.abs(want[o])))
+    assert not np.array_equal(np.delete(got, o), np.delete(fixed, o))
 
 
 # ------------------------------------------------------------------------------- selection variants

@@ -74,8 +74,19 @@ def test_plan_covers_every_tile_exactly_once(lib, rows, d, V, sms, cta_group):
     assert p["full_waves"] * p["group_m"] + p["rem_m"] == p["super_tiles"]
     if p["rem_m"]:
         assert 1 <= p["split_rem"] and p["rem_m"] * p["split_rem"] <= p["units"]
-    assert p["workspace_bytes"] == p["waves"] * p["grid"] * 2 * 3 * 128 * 4 + p["units"] * 8   # slots + progress words
-    assert p["workspace_bytes"] < 256 * rows + (1 << 20)              # never anything like rows x V
+    first = p["waves"] * p["grid"] * 2 * 3 * 128 * 4 + p["units"] * 8        # slots + progress words
+    if p["k_blocks"] <= p["chunk_kblocks"]:
+        assert p["workspace_bytes"] == first                      # one accumulation chunk: no second pass
+        assert first < 256 * rows + (1 << 20)                     # never anything like rows x V
+    else:
+        # adaptive chunks: control block, list and gathered hidden states of the rows to re-score (at most
+        # an eighth of the super tiles, 32 at most), and the second pass's own slots + progress words
+        up = lambda n: -(-n // 256) * 256
+        cap_rows = min(max(-(-p["super_tiles"] // 8), 1), 32, p["units"]) * 128 * cg
+        gathered = up(cap_rows * d * 2)
+        assert p["workspace_bytes"] == up(first) + 256 + up(cap_rows * 4) + gathered + up(first)
+        assert p["workspace_bytes"] - gathered < 512 * rows + (2 << 20)
+        assert gathered <= rows * d * 2 // 8 + 2 * 256 * d * 2
     covered = {}
     for w in range(p["waves"]):
         for c in range(p["grid"]):

@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import specs_oracle as O
 from paper_2506_15733_b200 import binding
 from paper_2506_15733_b200 import inputs as I
 from tests.gpu_util import BLK_RTOL, TOK_ATOL
@@ -50,9 +51,13 @@ def test_noalloc_matches_regular_entry_point_twice_in_a_row():
     # shared scratch (different plan, different slot count) and must not be affected by them
     cfg_a = I.StepConfig("na_a", 5100, 3, 5, (3, 40), 256, 2500, 0.05)
     cfg_b = I.StepConfig("na_b", 5101, 2, 4, (200, 200), 128, 1000, 0.08)
+    # a third one with a long reduction (d = 1024), where the regular entry point would by default lengthen
+    # its accumulation chunks; the allocation-free one always uses fixed 512-element chunks
+    cfg_c = I.StepConfig("na_d", 5103, 1, 3, (50, 90), 1024, 3000, 0.04)
     ctx = binding.Context(0)
+    ctx.set_accum_chunk(512)
     status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
-    for cfg in (cfg_a, cfg_b, cfg_a):
+    for cfg in (cfg_a, cfg_b, cfg_c, cfg_a):
         x, t = _device_inputs(cfg)
         want_tok, want_blk = _regular(ctx, t, x.rows, x.blocks)
         got_tok, got_blk = _noalloc(t, x.rows, x.blocks, status)
@@ -60,6 +65,11 @@ def test_noalloc_matches_regular_entry_point_twice_in_a_row():
         assert np.abs(got_tok - want_tok).max() <= TOK_ATOL
         assert np.all(np.abs(got_blk - want_blk) <= BLK_RTOL * np.abs(want_blk))
         assert np.array_equal(got_tok, want_tok)              # same kernels, same plan: in fact bit-identical
+        # and directly against the CPU oracle
+        oracle_tok = O.token_logprobs(x.hidden, x.w_vocab, x.token_ids)
+        oracle_blk = O.block_sums(oracle_tok, x.block_offsets)
+        assert np.abs(got_tok - oracle_tok).max() <= TOK_ATOL
+        assert np.all(np.abs(got_blk - oracle_blk) <= BLK_RTOL * np.abs(oracle_blk))
     assert int(status.item()) == 0
     assert ctx.device_status() == 0
     ctx.close()
