@@ -454,6 +454,34 @@ int specs_beam_step_host(specs_ctx* ctx,
                          float* h_tok_logprob, double* h_blk_logprob, float* h_weights,
                          int32_t* h_chosen, uint8_t* h_accept, void* cuda_stream);
 
+/* The same step in two halves, so that a caller can keep two steps in flight and
+ * have one step's copies run while the other step's kernels do (the paper runs the
+ * target's scoring and the PRM's concurrently, Appendix E.3; this is the same idea
+ * applied to the bus).  submit copies the small inputs into the context's pinned
+ * staging memory, enqueues the host-to-device copies on an internal copy stream, the
+ * kernels of specs_beam_step on `cuda_stream` behind them, and the device-to-host copy
+ * of the results on a second internal copy stream behind those; it returns a ticket
+ * without waiting for any of it.  wait blocks until that step's results have arrived
+ * and writes them to the output pointers given at submit.
+ *   - h_hidden is read by the copy engine after submit returns: it must stay valid and
+ *     unchanged until the matching wait, and only page-locked memory overlaps (the
+ *     driver stages pageable memory synchronously).  The other h_ inputs are consumed
+ *     before submit returns.  The output pointers must stay valid until wait.
+ *   - at most two steps may be in flight per context (a third submit returns
+ *     SPECS_ERR_LIMIT and enqueues nothing); each in-flight step owns one of the
+ *     context's two grow-only device arenas.  Waits may come in any order.
+ *   - wait returns SPECS_ERR_SHAPE for a ticket that is not in flight.
+ * specs_beam_step_host is submit followed by wait. */
+int specs_beam_step_host_submit(specs_ctx* ctx,
+                                const void* h_hidden, const void* W_vocab, const int32_t* h_token_ids,
+                                const int64_t* h_block_offsets, const int32_t* h_cand_offsets,
+                                const float* h_gen_tok_logprob, const float* h_reward, const float* h_uniforms,
+                                int64_t rows, int32_t d, int32_t V, int32_t B, int32_t P,
+                                float beta, float tau,
+                                float* h_tok_logprob, double* h_blk_logprob, float* h_weights,
+                                int32_t* h_chosen, uint8_t* h_accept, void* cuda_stream, int32_t* h_ticket);
+int specs_beam_step_host_wait(specs_ctx* ctx, int32_t ticket);
+
 /* Failure-detection self-test.  Every wait inside the scoring kernel is bounded: when
  * its time runs out it raises SPECS_DEV_TIMEOUT in the device status word and the
  * kernel winds down instead of hanging.  This call launches a one-CTA kernel that

@@ -77,6 +77,9 @@ SIGNATURES = {
     "specs_device_status": (C.c_int, [_vp, C.POINTER(C.c_uint32), _vp]),
     "specs_beam_step_host": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32,
                                        _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "specs_beam_step_host_submit": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i32, _i32, _i32,
+                                              _i32, _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp, C.POINTER(_i32)]),
+    "specs_beam_step_host_wait": (C.c_int, [_vp, _i32]),
     "specs_probe_wait_expiry": (C.c_int, [_vp, _i64, _vp]),
     "specs_set_timing": (C.c_int, [_vp, C.c_int]),
     "specs_score_kernel_ms": (C.c_float, [_vp, C.POINTER(_i32)]),
@@ -368,6 +371,26 @@ class Context:
             _ptr(h_gen_tok_logprob), _ptr(h_reward), _ptr(h_uniforms), rows, d, V, B, P, float(beta), float(tau),
             _ptr(h_tok_logprob), _ptr(h_blk_logprob), _ptr(h_weights), _ptr(h_chosen), _ptr(h_accept), _stream()),
             "specs_beam_step_host")
+
+    def specs_beam_step_host_submit(self, h_hidden, w_vocab, h_token_ids, h_block_offsets, h_cand_offsets,
+                                    h_gen_tok_logprob, h_reward, h_uniforms, beta, tau,
+                                    h_tok_logprob, h_blk_logprob, h_weights, h_chosen, h_accept) -> int:
+        """Enqueue one host-buffer step and return its ticket; the outputs are filled by ``..._wait(ticket)``.
+        The host arrays must stay alive and unchanged until then."""
+        rows, d = h_hidden.shape
+        V = w_vocab.shape[0]
+        B = h_block_offsets.shape[0] - 1
+        P = h_cand_offsets.shape[0] - 1
+        ticket = _i32(0)
+        _check(self._lib.specs_beam_step_host_submit(
+            self._h, _ptr(h_hidden), _ptr(w_vocab), _ptr(h_token_ids), _ptr(h_block_offsets), _ptr(h_cand_offsets),
+            _ptr(h_gen_tok_logprob), _ptr(h_reward), _ptr(h_uniforms), rows, d, V, B, P, float(beta), float(tau),
+            _ptr(h_tok_logprob), _ptr(h_blk_logprob), _ptr(h_weights), _ptr(h_chosen), _ptr(h_accept), _stream(),
+            C.byref(ticket)), "specs_beam_step_host_submit")
+        return int(ticket.value)
+
+    def specs_beam_step_host_wait(self, ticket: int):
+        _check(self._lib.specs_beam_step_host_wait(self._h, int(ticket)), "specs_beam_step_host_wait")
 
 
 class Policy(C.Structure):

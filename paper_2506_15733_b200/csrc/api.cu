@@ -126,8 +126,16 @@ int specs_destroy(specs_ctx* ctx) {
     if (!ctx) return SPECS_OK;
     DeviceGuard guard(ctx->device);
     for (auto& t : ctx->timed) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
-    if (ctx->arena) cudaFree(ctx->arena);
-    if (ctx->h_stage) cudaFreeHost(ctx->h_stage);
+    for (HostSlot& slot : ctx->host_slots) {
+        if (slot.ev_out && slot.busy) cudaEventSynchronize(slot.ev_out);
+        if (slot.arena) cudaFree(slot.arena);
+        if (slot.h_stage) cudaFreeHost(slot.h_stage);
+        if (slot.ev_in) cudaEventDestroy(slot.ev_in);
+        if (slot.ev_done) cudaEventDestroy(slot.ev_done);
+        if (slot.ev_out) cudaEventDestroy(slot.ev_out);
+    }
+    if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
+    if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
     if (ctx->d_status) cudaFree(ctx->d_status);
     delete ctx;
     return SPECS_OK;
@@ -635,13 +643,13 @@ float specs_score_kernel_ms(specs_ctx* ctx, int32_t* h_launches) {
     return mean;
 }
 
-int specs_beam_step_host(specs_ctx* ctx, const void* h_hidden, const void* W_vocab, const int32_t* h_token_ids,
-                         const int64_t* h_block_offsets, const int32_t* h_cand_offsets,
-                         const float* h_gen_tok_logprob, const float* h_reward, const float* h_uniforms,
-                         int64_t rows, int32_t d, int32_t V, int32_t B, int32_t P, float beta, float tau,
-                         float* h_tok_logprob, double* h_blk_logprob, float* h_weights, int32_t* h_chosen,
-                         uint8_t* h_accept, void* cuda_stream) {
-    if (!ctx) return SPECS_ERR_NULL;
+int specs_beam_step_host_submit(specs_ctx* ctx, const void* h_hidden, const void* W_vocab, const int32_t* h_token_ids,
+                                const int64_t* h_block_offsets, const int32_t* h_cand_offsets,
+                                const float* h_gen_tok_logprob, const float* h_reward, const float* h_uniforms,
+                                int64_t rows, int32_t d, int32_t V, int32_t B, int32_t P, float beta, float tau,
+                                float* h_tok_logprob, double* h_blk_logprob, float* h_weights, int32_t* h_chosen,
+                                uint8_t* h_accept, void* cuda_stream, int32_t* h_ticket) {
+    if (!ctx || !h_ticket) return SPECS_ERR_NULL;
     int st = check_score_shapes(rows, d, V, B);
     if (st != SPECS_OK) return st;
     if (P < 0) return SPECS_ERR_SHAPE;
@@ -654,6 +662,16 @@ int specs_beam_step_host(specs_ctx* ctx, const void* h_hidden, const void* W_voc
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return SPECS_ERR_CUDA;
+
+    HostSlot& slot = ctx->host_slots[ctx->next_ticket & 1u];
+    if (slot.busy) return SPECS_ERR_LIMIT;                   // two steps in flight at most: wait for the older one
+    if (!ctx->copy_in && (cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking) != cudaSuccess ||
+                          cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking) != cudaSuccess))
+        return SPECS_ERR_CUDA;
+    if (!slot.ev_in && (cudaEventCreateWithFlags(&slot.ev_in, cudaEventDisableTiming) != cudaSuccess ||
+                        cudaEventCreateWithFlags(&slot.ev_done, cudaEventDisableTiming) != cudaSuccess ||
+                        cudaEventCreateWithFlags(&slot.ev_out, cudaEventDisableTiming) != cudaSuccess))
+        return SPECS_ERR_CUDA;
 
     // Carve the arena (every piece 256-byte aligned): hidden states, then one block of the small inputs, then
     // one block of the outputs, then what never crosses the bus.  The two blocks are mirrored in a pinned
@@ -671,19 +689,20 @@ int specs_beam_step_host(specs_ctx* ctx, const void* h_hidden, const void* W_voc
     const size_t o_blk_g = carve((size_t)B * 8);
     const size_t ws_bytes = specs_score_workspace_bytes(ctx, rows, d, V);
     const size_t o_ws = carve(ws_bytes);
-    if (off > ctx->arena_bytes) {
-        if (ctx->arena) { cudaStreamSynchronize(stream); cudaFree(ctx->arena); ctx->arena = nullptr; ctx->arena_bytes = 0; }
-        if (cudaMalloc(&ctx->arena, off) != cudaSuccess) return SPECS_ERR_CUDA;
-        ctx->arena_bytes = off;
+    // the slot is idle (its last step was waited for), so its buffers may be replaced
+    if (off > slot.arena_bytes) {
+        if (slot.arena) { cudaFree(slot.arena); slot.arena = nullptr; slot.arena_bytes = 0; }
+        if (cudaMalloc(&slot.arena, off) != cudaSuccess) return SPECS_ERR_CUDA;
+        slot.arena_bytes = off;
     }
     const size_t stage_bytes = out1 - in0;
-    if (stage_bytes > ctx->stage_bytes) {
-        if (ctx->h_stage) { cudaStreamSynchronize(stream); cudaFreeHost(ctx->h_stage); ctx->h_stage = nullptr; ctx->stage_bytes = 0; }
-        if (cudaMallocHost(&ctx->h_stage, stage_bytes) != cudaSuccess) return SPECS_ERR_CUDA;
-        ctx->stage_bytes = stage_bytes;
+    if (stage_bytes > slot.stage_bytes) {
+        if (slot.h_stage) { cudaFreeHost(slot.h_stage); slot.h_stage = nullptr; slot.stage_bytes = 0; }
+        if (cudaMallocHost(&slot.h_stage, stage_bytes) != cudaSuccess) return SPECS_ERR_CUDA;
+        slot.stage_bytes = stage_bytes;
     }
-    uint8_t* A = static_cast<uint8_t*>(ctx->arena);
-    uint8_t* S = static_cast<uint8_t*>(ctx->h_stage) - in0;          // S + offset mirrors A + offset
+    uint8_t* A = static_cast<uint8_t*>(slot.arena);
+    uint8_t* S = static_cast<uint8_t*>(slot.h_stage) - in0;          // S + offset mirrors A + offset
     auto put = [&](size_t at, const void* src, size_t bytes) { if (src && bytes) std::memcpy(S + at, src, bytes); };
     put(o_ids, h_token_ids, (size_t)rows * 4);
     put(o_boff, h_block_offsets, (size_t)(B + 1) * 8);
@@ -691,10 +710,13 @@ int specs_beam_step_host(specs_ctx* ctx, const void* h_hidden, const void* W_voc
     put(o_gen, h_gen_tok_logprob, (size_t)rows * 4);
     put(o_rew, h_reward, (size_t)B * 4);
     put(o_uni, h_uniforms, (size_t)B * 4);
-    if (rows > 0 && cudaMemcpyAsync(A + o_hidden, h_hidden, (size_t)rows * d * 2, cudaMemcpyHostToDevice, stream) !=
-                        cudaSuccess)
+    // inputs on the inbound copy stream, kernels on the caller's stream, results on the outbound copy stream
+    if (rows > 0 && cudaMemcpyAsync(A + o_hidden, h_hidden, (size_t)rows * d * 2, cudaMemcpyHostToDevice,
+                                    ctx->copy_in) != cudaSuccess)
         return SPECS_ERR_CUDA;
-    if (cudaMemcpyAsync(A + in0, S + in0, out0 - in0, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    if (cudaMemcpyAsync(A + in0, S + in0, out0 - in0, cudaMemcpyHostToDevice, ctx->copy_in) != cudaSuccess ||
+        cudaEventRecord(slot.ev_in, ctx->copy_in) != cudaSuccess ||
+        cudaStreamWaitEvent(stream, slot.ev_in, 0) != cudaSuccess)
         return SPECS_ERR_CUDA;
 
     st = specs_beam_step(ctx, A + o_hidden, W_vocab, reinterpret_cast<int32_t*>(A + o_ids),
@@ -706,16 +728,52 @@ int specs_beam_step_host(specs_ctx* ctx, const void* h_hidden, const void* W_voc
                          reinterpret_cast<int32_t*>(A + o_cho), reinterpret_cast<uint8_t*>(A + o_acc), A + o_ws,
                          ws_bytes, cuda_stream);
     if (st != SPECS_OK) return st;
-    if (cudaMemcpyAsync(S + out0, A + out0, out1 - out0, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
-        cudaStreamSynchronize(stream) != cudaSuccess)
+    if (cudaEventRecord(slot.ev_done, stream) != cudaSuccess ||
+        cudaStreamWaitEvent(ctx->copy_out, slot.ev_done, 0) != cudaSuccess ||
+        cudaMemcpyAsync(S + out0, A + out0, out1 - out0, cudaMemcpyDeviceToHost, ctx->copy_out) != cudaSuccess ||
+        cudaEventRecord(slot.ev_out, ctx->copy_out) != cudaSuccess)
         return SPECS_ERR_CUDA;
-    auto get = [&](void* dst, size_t at, size_t bytes) { if (dst && bytes) std::memcpy(dst, S + at, bytes); };
-    get(h_tok_logprob, o_tok, (size_t)rows * 4);
-    get(h_blk_logprob, o_blk_t, (size_t)B * 8);
-    get(h_weights, o_wts, (size_t)B * 4);
-    get(h_chosen, o_cho, (size_t)P * 4);
-    get(h_accept, o_acc, (size_t)P);
+    slot.busy = true;
+    slot.ticket = ctx->next_ticket++;
+    slot.in0 = in0; slot.o_tok = o_tok; slot.o_blk = o_blk_t; slot.o_wts = o_wts; slot.o_cho = o_cho; slot.o_acc = o_acc;
+    slot.rows = rows; slot.B = B; slot.P = P;
+    slot.h_tok = h_tok_logprob; slot.h_blk = h_blk_logprob; slot.h_wts = h_weights; slot.h_cho = h_chosen;
+    slot.h_acc = h_accept;
+    *h_ticket = (int32_t)(slot.ticket & 0x7fffffffu);
     return SPECS_OK;
+}
+
+int specs_beam_step_host_wait(specs_ctx* ctx, int32_t ticket) {
+    if (!ctx) return SPECS_ERR_NULL;
+    HostSlot& slot = ctx->host_slots[(uint32_t)ticket & 1u];
+    if (!slot.busy || (int32_t)(slot.ticket & 0x7fffffffu) != ticket) return SPECS_ERR_SHAPE;   // no such step in flight
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return SPECS_ERR_CUDA;
+    slot.busy = false;
+    if (cudaEventSynchronize(slot.ev_out) != cudaSuccess) return SPECS_ERR_CUDA;
+    const uint8_t* S = static_cast<const uint8_t*>(slot.h_stage) - slot.in0;
+    auto get = [&](void* dst, size_t at, size_t bytes) { if (dst && bytes) std::memcpy(dst, S + at, bytes); };
+    get(slot.h_tok, slot.o_tok, (size_t)slot.rows * 4);
+    get(slot.h_blk, slot.o_blk, (size_t)slot.B * 8);
+    get(slot.h_wts, slot.o_wts, (size_t)slot.B * 4);
+    get(slot.h_cho, slot.o_cho, (size_t)slot.P * 4);
+    get(slot.h_acc, slot.o_acc, (size_t)slot.P);
+    return SPECS_OK;
+}
+
+int specs_beam_step_host(specs_ctx* ctx, const void* h_hidden, const void* W_vocab, const int32_t* h_token_ids,
+                         const int64_t* h_block_offsets, const int32_t* h_cand_offsets,
+                         const float* h_gen_tok_logprob, const float* h_reward, const float* h_uniforms,
+                         int64_t rows, int32_t d, int32_t V, int32_t B, int32_t P, float beta, float tau,
+                         float* h_tok_logprob, double* h_blk_logprob, float* h_weights, int32_t* h_chosen,
+                         uint8_t* h_accept, void* cuda_stream) {
+    int32_t ticket = 0;
+    const int st = specs_beam_step_host_submit(ctx, h_hidden, W_vocab, h_token_ids, h_block_offsets, h_cand_offsets,
+                                               h_gen_tok_logprob, h_reward, h_uniforms, rows, d, V, B, P, beta, tau,
+                                               h_tok_logprob, h_blk_logprob, h_weights, h_chosen, h_accept,
+                                               cuda_stream, &ticket);
+    if (st != SPECS_OK) return st;
+    return specs_beam_step_host_wait(ctx, ticket);
 }
 
 }  // extern "C"

@@ -469,6 +469,8 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
 
     bool compact = false;                                    // second pass: gathered rows rather than all rows
     if (kSecond) {
+        // the next kernel of the stream may set itself up from now on (it waits for this one's end itself)
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
         // the count is the merge kernel's: wait for it before anything else, and leave when there is no work
         asm volatile("griddepcontrol.wait;" ::: "memory");
         const uint32_t marked = *reinterpret_cast<const volatile uint32_t*>(&pass.ctl->count);
@@ -514,6 +516,8 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
     if (!kSecond) {
         // the kernel may have been launched while its predecessor in the stream still ran: wait for it here
         asm volatile("griddepcontrol.wait;" ::: "memory");
+        // ... and the merge kernel behind this one may be set up (it waits for this kernel's end itself)
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
         if (pass.ctl != nullptr && blockIdx.x == 0 && threadIdx.x == 0) pass.ctl->count = 0u;
     }
 

@@ -35,7 +35,9 @@ constexpr int kMergeBatch = 6;                              // splits whose six 
 // batch costs one trip to L2.
 struct RowFold { float max2; double sum2; float logit; bool marked; };
 
-__device__ __forceinline__ RowFold fold_row(const ScorePlan& plan, const float* __restrict__ workspace, int64_t row) {
+// The fold takes the splits first, first + step, ...: all of them by default, or a lane's share of them.
+__device__ __forceinline__ RowFold fold_row(const ScorePlan& plan, const float* __restrict__ workspace, int64_t row,
+                                            int first = 0, int step = 1) {
     const int mt = (int)(row / kBlockM), r = (int)(row % kBlockM);
     // the row tile's work unit: super tile (cta_group row tiles) and the CTA's rank inside the unit
     const int cg = plan.cta_group, sup = mt / cg, rank = mt % cg;
@@ -52,12 +54,12 @@ __device__ __forceinline__ RowFold fold_row(const ScorePlan& plan, const float* 
 
     RowFold f;
     f.max2 = -INFINITY; f.sum2 = 0.0; f.logit = -INFINITY; f.marked = false;
-    for (int s0 = 0; s0 < splits; s0 += kMergeBatch) {
+    for (int s0 = first; s0 < splits; s0 += kMergeBatch * step) {
         float v[kMergeBatch][6];
 #pragma unroll
         for (int u = 0; u < kMergeBatch; ++u) {
-            const bool live = s0 + u < splits;
-            const float* p = base + (size_t)(live ? s0 + u : s0) * stride;
+            const bool live = s0 + u * step < splits;
+            const float* p = base + (size_t)(live ? s0 + u * step : s0) * stride;
             const float m0 = __ldcg(p), s_0 = __ldcg(p + kBlockM), t0 = __ldcg(p + 2 * kBlockM);
             const float m1 = __ldcg(p + kHalf), s_1 = __ldcg(p + kHalf + kBlockM), t1 = __ldcg(p + kHalf + 2 * kBlockM);
             f.marked = f.marked || (live && (s_0 < 0.0f || s_1 < 0.0f));
@@ -76,6 +78,18 @@ __device__ __forceinline__ RowFold fold_row(const ScorePlan& plan, const float* 
             f.logit = fmaxf(f.logit, fmaxf(v[u][2], v[u][5]));
         }
     }
+    return f;
+}
+
+// Two folds over disjoint sets of splits into one.
+__device__ __forceinline__ RowFold combine_folds(const RowFold& a, const RowFold& b) {
+    RowFold f;
+    f.max2 = fmaxf(a.max2, b.max2);
+    f.sum2 = 0.0;
+    if (f.max2 != -INFINITY)
+        f.sum2 = a.sum2 * (double)exp2f(a.max2 - f.max2) + b.sum2 * (double)exp2f(b.max2 - f.max2);
+    f.logit = fmaxf(a.logit, b.logit);
+    f.marked = a.marked || b.marked;
     return f;
 }
 
@@ -101,8 +115,10 @@ struct CollectArgs {
     int32_t cap_rows;
 };
 constexpr int kMergeThreads = 128;
+constexpr int kMergeLanes = 4;                              // lanes that share a row's splits in merge_splits_kernel
+constexpr int kMergeRows = kMergeThreads / kMergeLanes;     // rows per CTA there
 
-// One thread per row: fold the first pass's splits and write the row's log-probability (or, for a holder
+// Four lanes per row, each folding every fourth split, then combined by shuffles: fold the first pass's splits and write the row's log-probability (or, for a holder
 // of one vocabulary shard, its partials: max in base-2 units, sum of 2^(x - max), drafted id's logit or
 // -inf, 0).  A marked row also takes the next place in the list of rows to re-score; then the CTA's
 // threads together copy the hidden states of the CTA's marked rows into the compact buffer.  Rows beyond
@@ -111,15 +127,27 @@ __global__ void __launch_bounds__(kMergeThreads)
 merge_splits_kernel(const ScorePlan plan, const float* __restrict__ workspace,
                     const int32_t* __restrict__ token_ids, float* __restrict__ tok_logprob,
                     float4* __restrict__ partials, const CollectArgs col, uint32_t* __restrict__ status) {
-    __shared__ int32_t marked_row[kMergeThreads], marked_at[kMergeThreads];
+    __shared__ int32_t marked_row[kMergeRows], marked_at[kMergeRows];
     __shared__ int marked_n;
-    asm volatile("griddepcontrol.wait;" ::: "memory");       // the scoring kernel's results
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (threadIdx.x == 0) marked_n = 0;
     __syncthreads();
-    const int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (row < plan.rows) {
-        const RowFold f = fold_row(plan, workspace, row);
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // the scoring kernel's results
+    const int sub = threadIdx.x % kMergeLanes;
+    // rows past the end fold row 0 (the shuffles below need every lane) and write nothing
+    const int64_t row_raw = (int64_t)blockIdx.x * kMergeRows + threadIdx.x / kMergeLanes;
+    const int64_t row = row_raw < plan.rows ? row_raw : 0;
+    RowFold f = fold_row(plan, workspace, row, sub, kMergeLanes);
+#pragma unroll
+    for (int o = 1; o < kMergeLanes; o <<= 1) {
+        RowFold g;
+        g.max2 = __shfl_xor_sync(kFull, f.max2, o);
+        g.sum2 = __shfl_xor_sync(kFull, f.sum2, o);
+        g.logit = __shfl_xor_sync(kFull, f.logit, o);
+        g.marked = __shfl_xor_sync(kFull, (int)f.marked, o) != 0;
+        f = combine_folds(f, g);
+    }
+    if (row_raw < plan.rows && sub == 0) {
         if (partials) partials[row] = make_float4(f.max2, (float)f.sum2, f.logit, 0.0f);
         else          tok_logprob[row] = fold_logprob(f, token_ids[row], plan.V, status);
         if (f.marked && col.ctl != nullptr) {
@@ -558,7 +586,7 @@ int launch_merge(specs_ctx* ctx, const ScorePlan& plan, void* workspace, const i
         col.row_bytes = plan.d * plan.elem_bytes;
         col.cap_rows = lay.cap_rows;
     }
-    const unsigned blocks = (unsigned)((plan.rows + kMergeThreads - 1) / kMergeThreads);
+    const unsigned blocks = (unsigned)((plan.rows + kMergeRows - 1) / kMergeRows);
     return launch_chained(merge_splits_kernel, blocks, kMergeThreads, stream, plan,
                           static_cast<const float*>(workspace), token_ids, tok_logprob,
                           reinterpret_cast<float4*>(partials), col, ctx->d_status);

@@ -173,6 +173,24 @@ struct FixView {
     int32_t cap_rows;
 };
 
+// One host-buffer step in flight: a grow-only device arena (hidden states, small inputs, outputs, scoring
+// workspace), a pinned mirror of the arena's small-input and output blocks, the events that order its copies
+// and kernels, and where its results go once it is waited for.
+struct HostSlot {
+    void* arena = nullptr;
+    size_t arena_bytes = 0;
+    void* h_stage = nullptr;
+    size_t stage_bytes = 0;
+    cudaEvent_t ev_in = nullptr, ev_done = nullptr, ev_out = nullptr;
+    bool busy = false;
+    uint32_t ticket = 0;
+    size_t in0 = 0, o_tok = 0, o_blk = 0, o_wts = 0, o_cho = 0, o_acc = 0;
+    int64_t rows = 0;
+    int32_t B = 0, P = 0;
+    float* h_tok = nullptr; double* h_blk = nullptr; float* h_wts = nullptr; int32_t* h_cho = nullptr;
+    uint8_t* h_acc = nullptr;
+};
+
 }  // namespace specs
 
 struct specs_ctx {
@@ -185,11 +203,10 @@ struct specs_ctx {
     int lead_tiles = 1;                    // see specs_set_tile_lead
     uint32_t* d_status = nullptr;          // device status word (SPECS_DEV_* bits)
     specs::EncodeTiledFn encode_tiled = nullptr;
-    // grow-only device arena for specs_beam_step_host
-    void* arena = nullptr;
-    size_t arena_bytes = 0;
-    void* h_stage = nullptr;               // pinned mirror of the arena's small-input and output blocks
-    size_t stage_bytes = 0;
+    // the host-buffer step: two slots, so that one step's copies run under the other's kernels
+    specs::HostSlot host_slots[2];
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;   // created on first use
+    uint32_t next_ticket = 0;
     std::vector<specs::CachedMap> maps;    // tensor maps of recent operands (round robin)
     size_t maps_next = 0;
     // optional per-launch timing of the tensor-core kernel

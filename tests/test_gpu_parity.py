@@ -380,6 +380,50 @@ def test_beam_step_host_equals_device_calls(ctx):
     assert e.value.status == 5
 
 
+def test_two_host_steps_in_flight_equal_two_serial_steps(ctx):
+    # two different steps submitted back to back (the second one's copies may run under the first one's
+    # kernels), waited for in both orders, against the same steps run one after the other
+    cfgs = [small_config("inflight_a", (3, 40), 3, 5, 256, 2500, seed=4910),
+            small_config("inflight_b", (10, 90), 2, 6, 1024, 3000, seed=4911)]    # the second has adaptive chunks
+    xs = [I.make_step_inputs(c) for c in cfgs]
+    w_devs = [binding.bf16_bits_to_device(x.w_vocab, "cuda:0") for x in xs]
+    pinned = [binding.bf16_bits_to_pinned(x.hidden) for x in xs]
+
+    def outputs(x):
+        P = len(x.cand_offsets) - 1
+        return [np.empty(x.rows, np.float32), np.empty(x.blocks, np.float64), np.empty(x.blocks, np.float32),
+                np.empty(P, np.int32), np.empty(P, np.uint8)]
+
+    serial = []
+    for x, w, h in zip(xs, w_devs, pinned):
+        o = outputs(x)
+        ctx.specs_beam_step_host(h, w, x.token_ids, x.block_offsets, x.cand_offsets, x.draft_tok_logprob, x.reward,
+                                 x.uniforms, 1.5, 0.55, *o)
+        serial.append(o)
+    for order in ((0, 1), (1, 0)):
+        outs = [outputs(x) for x in xs]
+        for o in outs:
+            for a in o:
+                a.fill(0)
+        tickets = [ctx.specs_beam_step_host_submit(h, w, x.token_ids, x.block_offsets, x.cand_offsets,
+                                                   x.draft_tok_logprob, x.reward, x.uniforms, 1.5, 0.55, *o)
+                   for x, w, h, o in zip(xs, w_devs, pinned, outs)]
+        assert tickets[0] != tickets[1]
+        with pytest.raises(binding.SpecsError) as e:          # a third step has no slot
+            ctx.specs_beam_step_host_submit(pinned[0], w_devs[0], xs[0].token_ids, xs[0].block_offsets,
+                                            xs[0].cand_offsets, xs[0].draft_tok_logprob, xs[0].reward,
+                                            xs[0].uniforms, 1.5, 0.55, *outputs(xs[0]))
+        assert e.value.status == 10
+        for k in order:
+            ctx.specs_beam_step_host_wait(tickets[k])
+            for got, want in zip(outs[k], serial[k]):
+                assert np.array_equal(got, want)
+        with pytest.raises(binding.SpecsError) as e:          # waited for already
+            ctx.specs_beam_step_host_wait(tickets[0])
+        assert e.value.status == 2
+    assert ctx.device_status() == 0
+
+
 # ------------------------------------------------------------------------------- adaptive accumulation chunks
 
 def _score_only(ctx, x):
