@@ -47,7 +47,8 @@ typedef enum specs_status {
     SPECS_ERR_CUDA = 7,            /* a CUDA runtime or driver call failed */
     SPECS_ERR_DEVICE_TIMEOUT = 8,  /* device status: a bounded wait in a kernel expired */
     SPECS_ERR_TOKEN_RANGE = 9,     /* device status: some drafted id was outside [0, V) */
-    SPECS_ERR_LIMIT = 10           /* a size exceeds a documented maximum */
+    SPECS_ERR_LIMIT = 10,          /* a size exceeds a documented maximum */
+    SPECS_ERR_DEVICE_BOUNDS = 11   /* device status (checked build only): a kernel met an index outside its buffer */
 } specs_status;
 
 /* Bits of the device status word returned by specs_device_status(). */
@@ -56,10 +57,22 @@ typedef enum specs_status {
 #define SPECS_DEV_ACCUM_RANGE  0x4u   /* informational: some rows were re-scored by the second pass, see
                                          specs_set_accum_chunk; does not change a return value */
 
+#define SPECS_DEV_BOUNDS       0x8u   /* checked build only: an index check inside a kernel failed; the access
+                                         was skipped (see specs_debug_build) */
+
+/* 1 if the library was compiled with -DSPECS_DEBUG (the checked build), else 0.  The checked build
+ * (libspecs_b200_debug.so; python -m paper_2506_15733_b200.build --debug) stands in for a memory
+ * checker: every kernel tests the indices of its global-memory accesses against the extents the host
+ * computed, skips an access that fails and raises SPECS_DEV_BOUNDS; it also contains the plain
+ * CUDA-core scoring engine SPECS_ENGINE_SIMT, a second GPU implementation for bisecting the
+ * tensor-core path.  Neither is in the default build. */
+int specs_debug_build(void);
+
 /* Scoring engines (see specs_set_engine). */
 #define SPECS_ENGINE_TCGEN05      0   /* tensor-core path: TMA + tcgen05.mma + TMEM, fused epilogue (default);
                                         the planner picks the tile shape (one CTA or a CTA pair per tile) */
-#define SPECS_ENGINE_SIMT         1   /* plain CUDA-core kernel; a bring-up and bisecting aid, never chosen automatically */
+#define SPECS_ENGINE_SIMT         1   /* plain CUDA-core kernel; a bring-up and bisecting aid in the checked build only
+                                        (specs_set_engine returns SPECS_ERR_SHAPE for it otherwise) */
 #define SPECS_ENGINE_TCGEN05_1CTA 2   /* tensor-core path, forced to 128-row tiles run by single CTAs */
 #define SPECS_ENGINE_TCGEN05_2CTA 3   /* tensor-core path, forced to 256-row tiles run by CTA pairs
                                         (tcgen05.mma.cta_group::2; each CTA stages half of the W tile) */
@@ -426,6 +439,11 @@ int specs_controller_generators(const specs_controller* ctrl, int32_t* h_gen);
  * ignored where h_chosen < 0), h_uniforms float [P] (SPECS_POLICY_RANDOM only, else may be NULL). */
 int specs_controller_advance(specs_controller* ctrl, const int32_t* h_chosen, const uint8_t* h_flag,
                              const int64_t* h_chosen_len, const float* h_uniforms);
+/* h_appended uint8 [P] out: 1 where the last specs_controller_advance appended the problem's
+ * selected block to its trace (Algorithm 1, Step II), 0 where it did not (problem finished,
+ * nothing selected, or an RSD++ draft step that the target redoes).  The caller's copy of the
+ * trace follows this, not its own reading of the policy. */
+int specs_controller_appended(const specs_controller* ctrl, uint8_t* h_appended);
 /* Per problem, each int64 [P] out and optional: appended tokens, appended blocks, appended
  * blocks that the target generated, generation rounds the target ran (RSD++ retries count). */
 int specs_controller_stats(const specs_controller* ctrl, int64_t* h_length, int64_t* h_steps,
@@ -433,8 +451,8 @@ int specs_controller_stats(const specs_controller* ctrl, int64_t* h_length, int6
 
 /* Synchronise `cuda_stream`, return the device status word (a combination of
  * SPECS_DEV_* bits, 0 if clean) through *h_bits and clear it.  Returns
- * SPECS_ERR_DEVICE_TIMEOUT / SPECS_ERR_TOKEN_RANGE (timeout first) when a bit is
- * set, SPECS_OK otherwise.  h_bits may be NULL. */
+ * SPECS_ERR_DEVICE_TIMEOUT / SPECS_ERR_DEVICE_BOUNDS / SPECS_ERR_TOKEN_RANGE (the first
+ * of these whose bit is set), SPECS_OK otherwise.  h_bits may be NULL. */
 int specs_device_status(specs_ctx* ctx, uint32_t* h_bits, void* cuda_stream);
 
 /* One whole beam step from HOST buffers (the end-to-end path): copies the step's

@@ -80,8 +80,17 @@ const char* specs_status_string(int status) {
         case SPECS_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel expired";
         case SPECS_ERR_TOKEN_RANGE: return "a drafted token id was outside [0, V)";
         case SPECS_ERR_LIMIT: return "a size exceeds a documented maximum";
+        case SPECS_ERR_DEVICE_BOUNDS: return "an index check inside a kernel failed (checked build)";
         default: return "unknown status";
     }
+}
+
+int specs_debug_build(void) {
+#ifdef SPECS_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
 }
 
 int specs_create(specs_ctx** out, int device) {
@@ -146,6 +155,9 @@ int specs_set_engine(specs_ctx* ctx, int engine) {
     if (engine != SPECS_ENGINE_TCGEN05 && engine != SPECS_ENGINE_SIMT && engine != SPECS_ENGINE_TCGEN05_1CTA &&
         engine != SPECS_ENGINE_TCGEN05_2CTA)
         return SPECS_ERR_SHAPE;
+#ifndef SPECS_DEBUG
+    if (engine == SPECS_ENGINE_SIMT) return SPECS_ERR_SHAPE;     // the bisecting aid exists in the checked build only
+#endif
     if (engine == SPECS_ENGINE_TCGEN05_2CTA && ctx->pair_units <= 0) return SPECS_ERR_CUDA;
     ctx->engine = engine;
     return SPECS_OK;
@@ -227,10 +239,13 @@ int specs_score_blocks(specs_ctx* ctx, const void* hidden, const void* W_vocab, 
     if (!guard.ok) return SPECS_ERR_CUDA;
 
     if (rows > 0) {
+#ifdef SPECS_DEBUG
         if (ctx->engine == SPECS_ENGINE_SIMT) {
             st = launch_score_simt(ctx, hidden, W_vocab, token_ids, rows, d, V, tok_logprob, stream);
             if (st != SPECS_OK) return st;
-        } else {
+        } else
+#endif
+        {
             const int cta_group = ctx->engine == SPECS_ENGINE_TCGEN05_1CTA ? 1
                                 : ctx->engine == SPECS_ENGINE_TCGEN05_2CTA ? 2 : kCtaGroupAuto;
             const ScorePlan plan = make_score_plan(rows, d, V, ctx->num_sms, ctx->pair_units, cta_group,
@@ -601,6 +616,7 @@ int specs_device_status(specs_ctx* ctx, uint32_t* h_bits, void* cuda_stream) {
         return SPECS_ERR_CUDA;
     if (h_bits) *h_bits = bits;
     if (bits & SPECS_DEV_TIMEOUT) return SPECS_ERR_DEVICE_TIMEOUT;
+    if (bits & SPECS_DEV_BOUNDS) return SPECS_ERR_DEVICE_BOUNDS;
     if (bits & SPECS_DEV_TOKEN_RANGE) return SPECS_ERR_TOKEN_RANGE;
     return SPECS_OK;
 }

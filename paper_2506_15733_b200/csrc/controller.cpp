@@ -15,6 +15,7 @@ struct specs_controller {
     int32_t problems;
     std::vector<int32_t> gen;              // model that drafts the next step
     std::vector<int64_t> length, steps, target_steps, target_calls;
+    std::vector<uint8_t> appended;         // whether the last advance() appended the problem's selected block
 
     bool done(int32_t p) const { return length[p] >= policy.target_len || steps[p] >= policy.max_steps; }
 };
@@ -39,6 +40,7 @@ int specs_controller_create(specs_controller** out, int32_t P, const specs_polic
     c->steps.assign(P, 0);
     c->target_steps.assign(P, 0);
     c->target_calls.assign(P, 0);
+    c->appended.assign(P, 0);
     *out = c;
     return SPECS_OK;
 }
@@ -63,6 +65,7 @@ int specs_controller_advance(specs_controller* c, const int32_t* h_chosen, const
     for (int32_t p = 0; p < c->problems; ++p)
         if (!c->done(p) && h_chosen[p] >= 0 && h_chosen_len[p] < 0) return SPECS_ERR_SHAPE;
     for (int32_t p = 0; p < c->problems; ++p) {
+        c->appended[p] = 0;
         if (c->done(p)) continue;
         const int32_t g = c->gen[p];
         if (g == SPECS_GEN_TARGET) ++c->target_calls[p];
@@ -73,6 +76,7 @@ int specs_controller_advance(specs_controller* c, const int32_t* h_chosen, const
         if (h_chosen[p] >= 0) {                    // append the selected block
             c->length[p] += h_chosen_len[p];
             ++c->steps[p];
+            c->appended[p] = 1;
             if (g == SPECS_GEN_TARGET) ++c->target_steps[p];
         }
         switch (c->policy.policy) {
@@ -94,6 +98,12 @@ int specs_controller_advance(specs_controller* c, const int32_t* h_chosen, const
                 break;
         }
     }
+    return SPECS_OK;
+}
+
+int specs_controller_appended(const specs_controller* c, uint8_t* h_appended) {
+    if (!c || (!h_appended && c->problems > 0)) return SPECS_ERR_NULL;
+    for (int32_t p = 0; p < c->problems; ++p) h_appended[p] = c->appended[p];
     return SPECS_OK;
 }
 

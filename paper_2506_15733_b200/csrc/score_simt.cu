@@ -2,6 +2,8 @@
 // computing each logit as an fp32 dot product and keeping an online (max, sum-exp, drafted
 // logit) state.  It exists to bring the library up and to bisect the tensor-core path on sizes
 // the CPU cannot check quickly; it is selected only by an explicit specs_set_engine() call.
+// Compiled into the checked build (-DSPECS_DEBUG) only.
+#ifdef SPECS_DEBUG
 #include <cuda_bf16.h>
 
 #include "specs_internal.h"
@@ -91,3 +93,4 @@ int launch_score_simt(specs_ctx* ctx, const void* hidden, const void* w_vocab, c
 }
 
 }  // namespace specs
+#endif  // SPECS_DEBUG

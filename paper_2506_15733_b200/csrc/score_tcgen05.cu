@@ -550,7 +550,8 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
             for (int n = nb; n < ne && ok; ++n) {
                 if (pace && gm_w > 1) {
                     const int t = n - nb;
-                    if (lane == 0) st_progress(progress + unit, pace_key(plan.epoch, w, t));
+                    if (lane == 0 && SPECS_IN_BOUNDS(unit, plan.units, status))
+                        st_progress(progress + unit, pace_key(plan.epoch, w, t));
                     if (t >= plan.lead_tiles) {
                         const unsigned long long need = pace_key(plan.epoch, w, t - plan.lead_tiles);
                         const unsigned long long t0 = global_timer_ns();
@@ -717,9 +718,12 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
             float assumed = INFINITY;                        // magnitude the lengthened chunks were sized for
             const int64_t row = (int64_t)(st * kCg + (int)rank) * kBlockM + row_in_tile;
             // the row of the caller's arrays behind this one: itself, or the marked row gathered here
-            const int64_t src = (kSecond && compact && row < plan.rows) ? (int64_t)pass.list[row] : row;
+            int64_t src = row;
+            if (kSecond && compact && row < plan.rows && SPECS_IN_BOUNDS(row, pass.cap_rows, status))
+                src = (int64_t)pass.list[row];
             // ids are indices into the whole vocabulary; this W holds rows id_offset .. id_offset + V - 1
-            const int32_t id = (row < plan.rows) ? token_ids[src] - plan.id_offset : -1;
+            const int32_t id = (row < plan.rows && SPECS_IN_BOUNDS(src, plan_in.rows, status))
+                                   ? token_ids[src] - plan.id_offset : -1;
             float row_scale = 0.0f;
             if (kFp8 && row < plan.rows) row_scale = (kSecond && compact) ? pass.scale_compact[row] : hidden_scale[src];
             // state in base-2 units: run_max = max(z) * log2(e), run_sum = sum 2^(z*log2e - run_max)
@@ -843,10 +847,13 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                 const bool over = run_sum > 0.0f && (fabsf(run_max) > assumed * kLog2e ||
                                                      (picked != -INFINITY && fabsf(picked) > assumed));
                 if (__any_sync(0xffffffffu, over) && lane == 0) atomicOr(status, SPECS_DEV_ACCUM_RANGE);
-                float* slot = workspace + ((size_t)w * plan.grid + cta) * kTripleFloats + half * 3 * kBlockM;
-                slot[row_in_tile] = run_max;
-                slot[kBlockM + row_in_tile] = over ? -run_sum : run_sum;
-                slot[2 * kBlockM + row_in_tile] = picked;
+                const size_t at = ((size_t)w * plan.grid + cta) * kTripleFloats + half * 3 * kBlockM;
+                float* slot = workspace + at;
+                if (SPECS_IN_BOUNDS(at + 2 * kBlockM + row_in_tile, plan_slot_bytes(plan) / sizeof(float), status)) {
+                    slot[row_in_tile] = run_max;
+                    slot[kBlockM + row_in_tile] = over ? -run_sum : run_sum;
+                    slot[2 * kBlockM + row_in_tile] = picked;
+                }
             }
         }
     }

@@ -37,7 +37,7 @@ struct RowFold { float max2; double sum2; float logit; bool marked; };
 
 // The fold takes the splits first, first + step, ...: all of them by default, or a lane's share of them.
 __device__ __forceinline__ RowFold fold_row(const ScorePlan& plan, const float* __restrict__ workspace, int64_t row,
-                                            int first = 0, int step = 1) {
+                                            int first = 0, int step = 1, uint32_t* status = nullptr) {
     const int mt = (int)(row / kBlockM), r = (int)(row % kBlockM);
     // the row tile's work unit: super tile (cta_group row tiles) and the CTA's rank inside the unit
     const int cg = plan.cta_group, sup = mt / cg, rank = mt % cg;
@@ -54,6 +54,11 @@ __device__ __forceinline__ RowFold fold_row(const ScorePlan& plan, const float* 
 
     RowFold f;
     f.max2 = -INFINITY; f.sum2 = 0.0; f.logit = -INFINITY; f.marked = false;
+    // checked build: the last float this row's fold reads must lie inside the plan's slots
+    if (status != nullptr && splits > 0 &&
+        !SPECS_IN_BOUNDS((base - workspace) + (size_t)(splits - 1) * stride + kHalf + 2 * kBlockM,
+                         plan_slot_bytes(plan) / sizeof(float), status))
+        return f;
     for (int s0 = first; s0 < splits; s0 += kMergeBatch * step) {
         float v[kMergeBatch][6];
 #pragma unroll
@@ -137,7 +142,7 @@ merge_splits_kernel(const ScorePlan plan, const float* __restrict__ workspace,
     // rows past the end fold row 0 (the shuffles below need every lane) and write nothing
     const int64_t row_raw = (int64_t)blockIdx.x * kMergeRows + threadIdx.x / kMergeLanes;
     const int64_t row = row_raw < plan.rows ? row_raw : 0;
-    RowFold f = fold_row(plan, workspace, row, sub, kMergeLanes);
+    RowFold f = fold_row(plan, workspace, row, sub, kMergeLanes, status);
 #pragma unroll
     for (int o = 1; o < kMergeLanes; o <<= 1) {
         RowFold g;
@@ -168,6 +173,8 @@ merge_splits_kernel(const ScorePlan plan, const float* __restrict__ workspace,
     for (int k = 0; k < n; ++k) {
         const uint4* src = reinterpret_cast<const uint4*>(col.hidden + (size_t)marked_row[k] * col.row_bytes);
         uint4* dst = reinterpret_cast<uint4*>(col.compact + (size_t)marked_at[k] * col.row_bytes);
+        if (!SPECS_IN_BOUNDS(marked_at[k], col.cap_rows, status) || !SPECS_IN_BOUNDS(marked_row[k], plan.rows, status))
+            continue;
         for (int v = threadIdx.x; v < vecs; v += kMergeThreads) dst[v] = __ldg(src + v);
     }
 }
@@ -196,7 +203,8 @@ fix_merge_kernel(const ScorePlan plan, const FixView fix, const int32_t* __restr
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     const int64_t row = compact ? (int64_t)fix.list[i] : i;
-    const RowFold f = fold_row(plan2, fix.slots, i);
+    const RowFold f = fold_row(plan2, fix.slots, i, 0, 1, status);
+    if (!SPECS_IN_BOUNDS(row, plan.rows, status)) return;
     if (partials) partials[row] = make_float4(f.max2, (float)f.sum2, f.logit, 0.0f);
     else          tok_logprob[row] = fold_logprob(f, token_ids[row], plan.V, status);
 }
@@ -435,11 +443,11 @@ __device__ __forceinline__ void apply_second_pass(const ScorePlan& plan, const F
         for (int i = tid; i < n; i += nthreads) {
             const int64_t row = fix.list[i];
             if (row >= row_a && row < row_b)
-                tok[row] = fold_logprob(fold_row(plan2, fix.slots, i), token_ids[row], plan.V, status);
+                tok[row] = fold_logprob(fold_row(plan2, fix.slots, i, 0, 1, status), token_ids[row], plan.V, status);
         }
     } else {
         for (int64_t row = row_a + tid; row < row_b; row += nthreads)
-            tok[row] = fold_logprob(fold_row(plan2, fix.slots, row), token_ids[row], plan.V, status);
+            tok[row] = fold_logprob(fold_row(plan2, fix.slots, row, 0, 1, status), token_ids[row], plan.V, status);
     }
 }
 

@@ -13,6 +13,21 @@
 
 namespace specs {
 
+// ---- index checks of the checked build (-DSPECS_DEBUG) ------------------------------------------
+// SPECS_IN_BOUNDS(index, extent, status) is true when 0 <= index < extent.  In the checked build a
+// failing index raises SPECS_DEV_BOUNDS in the status word and the caller skips the access; in the
+// default build the macro is the constant true and costs nothing.
+#ifdef SPECS_DEBUG
+__device__ __forceinline__ bool index_in_bounds(int64_t index, int64_t extent, uint32_t* status) {
+    if (index >= 0 && index < extent) return true;
+    atomicOr(status, SPECS_DEV_BOUNDS);
+    return false;
+}
+#define SPECS_IN_BOUNDS(index, extent, status) ::specs::index_in_bounds((int64_t)(index), (int64_t)(extent), (status))
+#else
+#define SPECS_IN_BOUNDS(index, extent, status) true
+#endif
+
 // ---- tile geometry of the tensor-core scoring kernel -----------------------------------------
 constexpr int kBlockM = 128;   // drafted rows per tile   (= TMEM lanes, one epilogue thread per row)
 constexpr int kBlockN = 256;   // vocabulary entries per tile (= fp32 TMEM columns of one accumulator)

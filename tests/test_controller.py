@@ -31,8 +31,11 @@ def test_native_controller_tracks_the_oracle(policy, sticky):
         flag = (rng.random(P) < 0.4).astype(np.uint8)
         lens = rng.integers(1, 40, P).astype(np.int64)
         u = I.draw_uniforms(6700 + k, P)
+        steps_before = list(want.steps)
         want.advance(chosen, flag, lens, u)
         got.advance(chosen, flag, lens, u)
+        # the controller says which problems appended their selected block in this update
+        assert got.appended().tolist() == [int(a != b) for a, b in zip(want.steps, steps_before)]
     st = got.stats()
     assert st["length"].tolist() == want.length and st["steps"].tolist() == want.steps
     assert st["target_steps"].tolist() == want.target_steps and st["target_calls"].tolist() == want.target_calls

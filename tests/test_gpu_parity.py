@@ -34,9 +34,11 @@ def small_config(name, rows_per_block, problems, beams, d, V, seed, **kw):
 # ------------------------------------------------------------------------------- tiny, both engines
 
 TC_ENGINES = [binding.ENGINE_TCGEN05_1CTA, binding.ENGINE_TCGEN05_2CTA]   # both tile shapes of the tensor-core kernel
+# the plain CUDA-core engine exists in the checked build only (SPECS_B200_DEBUG=1, see tests/test_gpu_debug_build.py)
+SIMT_ENGINE = [binding.ENGINE_SIMT] if binding.debug_build() else []
 
 
-@pytest.mark.parametrize("engine", [binding.ENGINE_SIMT, binding.ENGINE_TCGEN05] + TC_ENGINES)
+@pytest.mark.parametrize("engine", SIMT_ENGINE + [binding.ENGINE_TCGEN05] + TC_ENGINES)
 def test_tiny_config_full_step(ctx, engine):
     x = I.make_step_inputs(I.CONFIGS["tiny"])
     ctx.set_engine(engine)
@@ -142,7 +144,7 @@ def test_out_of_range_token_is_nan_and_flagged(ctx):
     x.token_ids = x.token_ids.copy()
     x.token_ids[3] = 300
     x.token_ids[9] = -2
-    for engine in (binding.ENGINE_TCGEN05_1CTA, binding.ENGINE_TCGEN05_2CTA, binding.ENGINE_SIMT):
+    for engine in TC_ENGINES + SIMT_ENGINE:
         ctx.set_engine(engine)
         try:
             s = DeviceStep(ctx, x)
@@ -1007,3 +1009,69 @@ def test_run_specs_helper_follows_the_controller(ctx):
                 assert int(ref["chosen"][j]) in match
             pos[p] += int(lens[match[0]]) if int(ref["chosen"][j]) not in match else int(lens[int(ref["chosen"][j])])
     assert ctx.device_status() == 0
+
+
+@pytest.mark.parametrize("policy,select_rule", [(binding.POLICY_RSD, None), (binding.POLICY_DRAFT_START, None),
+                                                (binding.POLICY_RANDOM, None),
+                                                (binding.POLICY_ONLY_DRAFT, binding.SELECT_BEST_REWARD)])
+def test_run_specs_dispatches_every_policy_like_the_oracle_loop(ctx, policy, select_rule):
+    # The packaged loop under the policies of the baselines and ablations, replayed on the CPU with the
+    # oracle's selection, switch rules and controller.  Rewards are spaced by 0.04 and beta is large, so
+    # every pick is decided by a wide margin and both loops must agree step by step.
+    from paper_2506_15733_b200 import loop as LP
+    P, n, d, Vv, beta, tau = 3, 4, 64, 500, 1000.0, 0.6
+    w_bits = I.make_step_inputs(small_config("loop_w", (1, 1), 1, 1, d, Vv, seed=5500)).w_vocab
+    w_dev = binding.bf16_bits_to_device(w_bits, "cuda:0")
+    asked, batches = [], []
+
+    def draft_fn(gens, live):
+        step = len(asked)
+        asked.append(gens.copy())
+        x = I.make_step_inputs(small_config("loop", (4, 12), len(live), n, d, Vv, seed=6400 + 10 * policy + step))
+        x.w_vocab = w_bits
+        perm = np.random.Generator(np.random.Philox(key=[6450, step])).permutation(n)
+        for j, p in enumerate(live):
+            lo = 0.62 if gens[p] == binding.GEN_TARGET else (0.40 if (step + p) % 2 else 0.55)
+            x.reward[j * n:(j + 1) * n] = (lo + 0.04 * perm).astype(np.float32)
+        s = DeviceStep(ctx, x)
+        batches.append((x, live.copy()))
+        return LP.DraftBatch(s.hidden, s.token_ids, s.block_offsets, s.cand_offsets, s.reward, s.uniforms, s.draft)
+
+    uni = lambda it: I.draw_uniforms(7000 + it, P)
+    ctl = binding.Controller(P, policy, target_len=40, p_target=0.5)
+    res = LP.run_specs(ctx, ctl, draft_fn, w_dev, beta, tau, max_block_len=16, max_iters=60,
+                       select_rule=select_rule, switch_uniforms=uni if policy == binding.POLICY_RANDOM else None)
+    assert (ctl.generators() == binding.GEN_DONE).all()
+
+    rule = OV.SELECT_BEST_REWARD if policy == binding.POLICY_RSD or select_rule == binding.SELECT_BEST_REWARD \
+        else OV.SELECT_SUBSAMPLE
+    switch = {binding.POLICY_DRAFT_START: OV.SWITCH_NONE_ABOVE, binding.POLICY_RSD: OV.SWITCH_CHOSEN_BELOW}.get(
+        policy, OV.SWITCH_ANY_ABOVE)
+    want_ctl = OV.Controller(P, policy, target_len=40, p_target=0.5)
+    want_traces = [[] for _ in range(P)]
+    for it, ((x, live), gens) in enumerate(zip(batches, asked)):
+        assert gens.tolist() == want_ctl.generators()
+        LP_t = O.block_sums(O.token_logprobs(x.hidden, x.w_vocab, x.token_ids), x.block_offsets)
+        LQ = O.block_sums(x.draft_tok_logprob, x.block_offsets)
+        c, w, margin = OV.select(LP_t, LQ, x.reward, None, x.cand_offsets, beta, x.uniforms, rule)
+        assert np.all(margin > (0.03 if rule == OV.SELECT_BEST_REWARD else 1.0))   # rewards 0.04 apart; beta * 0.04 = 40
+        f = OV.switch_flags(x.reward, x.cand_offsets, c, tau, switch)
+        chosen = np.full(P, -1, np.int32); flag = np.zeros(P, np.uint8); clen = np.zeros(P, np.int64)
+        for j, p in enumerate(live):
+            a = int(x.cand_offsets[j]) + int(c[j])
+            chosen[p], flag[p] = c[j], f[j]
+            clen[p] = x.block_offsets[a + 1] - x.block_offsets[a]
+        before = list(want_ctl.steps)
+        want_ctl.advance(chosen, flag, clen, uni(it))
+        for j, p in enumerate(live):
+            if want_ctl.steps[p] != before[p]:
+                a = int(x.cand_offsets[j]) + int(c[j])
+                want_traces[p].extend(x.token_ids[x.block_offsets[a]:x.block_offsets[a + 1]].tolist())
+    assert res.traces == want_traces
+    st = ctl.stats()
+    assert st["length"].tolist() == want_ctl.length == [len(t) for t in res.traces]
+    assert st["steps"].tolist() == want_ctl.steps and st["target_calls"].tolist() == want_ctl.target_calls
+    if policy == binding.POLICY_RSD:
+        assert sum(st["target_calls"]) > 0 and sum(st["target_steps"]) < sum(st["steps"])   # both routes were taken
+    assert ctx.device_status() == 0
+

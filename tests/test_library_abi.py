@@ -124,3 +124,35 @@ def test_planner_prefers_pairs_except_for_a_single_row_tile(lib):
     assert binding.score_plan(65536, 3584, 151936, 148)["cta_group"] == 2
     assert binding.score_plan(100, 3584, 151936, 148)["cta_group"] == 1     # 256-row tiles would be half empty
     assert binding.score_plan(1024, 3584, 151936, 1)["cta_group"] == 1      # no pair fits on one SM
+
+
+def test_binding_checks_tensor_arguments_before_the_call():
+    import numpy as np
+    # what the C ABI cannot see from a bare pointer: element type, contiguity, size, device
+    import torch
+    ok = torch.zeros(8, dtype=torch.int32)
+    assert binding.device_arg(None, "i32", 8, 0, "x") is None
+    with pytest.raises(TypeError):
+        binding.device_arg(ok.to(torch.int64), "i32", 8, 0, "token_ids")          # int64 ids
+    with pytest.raises(TypeError):
+        binding.device_arg(np.zeros(8, np.int32), "i32", 8, 0, "token_ids")        # not a tensor
+    with pytest.raises(ValueError):
+        binding.device_arg(torch.zeros((4, 4), dtype=torch.bfloat16)[:, :2], "bf16", 8, 0, "hidden")   # a slice
+    with pytest.raises(ValueError):
+        binding.device_arg(ok, "i32", 9, 0, "tok_logprob")                        # too short
+    with pytest.raises(ValueError):
+        binding.device_arg(ok, "i32", 8, 0, "token_ids")                          # a host tensor
+
+
+def test_checked_build_exports_the_same_symbols_and_says_what_it_is(lib):
+    import ctypes
+    from paper_2506_15733_b200 import build
+    assert lib.specs_debug_build() == (1 if binding.debug_build() else 0)
+    if not os.path.exists(build.LIB_PATH_DEBUG):
+        pytest.skip("checked library not built")
+    dbg = ctypes.CDLL(build.LIB_PATH_DEBUG)
+    for name in binding.SIGNATURES:
+        assert hasattr(dbg, name), name
+    dbg.specs_debug_build.restype = ctypes.c_int
+    assert dbg.specs_debug_build() == 1
+
