@@ -228,7 +228,7 @@ class Workload:
         self.chosen = torch.empty(P, dtype=torch.int32, device=dev)
         self.accept = torch.empty(P, dtype=torch.uint8, device=dev)
         self.plan = binding.score_plan(rows, d, V, ctx.sm_count())
-        two_pass = self.plan["k_blocks"] > self.plan["chunk_kblocks"]
+        two_pass = self.plan["k_blocks"] > self.plan["chunk_kblocks"] and self.plan["row_tiles"] > 1
         # score tiles; merge of the vocabulary splits; second pass (adaptive chunks only); finish (block sums,
         # SubSample + switch)
         self.launches_per_step = 4 if two_pass else 3
@@ -443,6 +443,9 @@ def main():
     ap.add_argument("--fp8", action="store_true",
                     help="time the E4M3 variant instead (reduced precision: not the headline; W quantised once, "
                          "hidden states quantised inside every step)")
+    ap.add_argument("--problems", type=int, default=None,
+                    help="shrink the workload to this many problems (same recipe; for profiler captures, whose "
+                         "size must stay small; the line's config then carries the reduced counts)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-per-config", action="store_true", help="measure the headline workload only")
@@ -456,6 +459,8 @@ def main():
         return                                               # rank 0 alone times the CPU oracle
     from paper_2506_15733_b200 import inputs
     cfg = inputs.CONFIGS[args.config]
+    if args.problems is not None:
+        cfg = inputs.scaled(cfg, problems=int(args.problems))
 
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else args.steps
@@ -600,7 +605,7 @@ def launches_of(binding, x, cfg, ctx, fp8) -> int:
     """Kernels of this library launched per step: score tiles, merge, finish, plus the second scoring pass
     when the plan has adaptive accumulation chunks, plus the quantisation of the hidden states for E4M3."""
     p = binding.score_plan(x.rows, cfg.d, cfg.vocab, ctx.sm_count())
-    return 3 + (1 if p["k_blocks"] > p["chunk_kblocks"] else 0) + (1 if fp8 else 0)
+    return 3 + (1 if p["k_blocks"] > p["chunk_kblocks"] and p["row_tiles"] > 1 else 0) + (1 if fp8 else 0)
 
 
 if __name__ == "__main__":

@@ -70,7 +70,9 @@ ScorePlan make_score_plan(int64_t rows, int32_t d, int32_t V, int32_t num_sms, i
     const int32_t k_elems = kBlockK * 2 / elem_bytes;        // elements in a 128-byte k-block
     p.k_blocks = (d + k_elems - 1) / k_elems;
     p.chunk_kblocks = (chunk_kblocks > 0 && chunk_kblocks < p.k_blocks) ? chunk_kblocks : p.k_blocks;
-    p.adaptive = (adaptive && p.chunk_kblocks < p.k_blocks) ? 1 : 0;
+    // A single row tile (at most 128 rows) is bound by streaming W from HBM, not by the tensor pipe: the
+    // restarts of short accumulation chunks cost it nothing, so it keeps the base chunks and needs no second pass.
+    p.adaptive = (adaptive && p.chunk_kblocks < p.k_blocks && p.row_tiles > 1) ? 1 : 0;
     if (pair_units <= 0 && cta_group == 2) cta_group = 1;      // pairs unavailable on this device
     if (cta_group == 1 || pair_units <= 0) {
         fill_plan(&p, 1, num_sms);

@@ -94,13 +94,16 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
 constexpr unsigned long long kDrainLimitNs = 20000000ull;    // 20 ms per stage when draining after an abort
 constexpr float kLog2e = 1.4426950408889634f;
 
+constexpr size_t kControlBytes = 5120;                   // barriers, published magnitudes, staged column scales
+constexpr int kScaleBufs = 4;                            // vocabulary tiles whose column scales are staged at once
+
 // Per tile shape: W rows staged per CTA and k-block, stage size, ring depth, shared memory.
 template <int kCg> struct Shape {
     static constexpr int kBRows = kBlockN / kCg;                         // 256, or this CTA's half
     static constexpr uint32_t kBBytes = kBRows * kBlockK * 2;            // 32 KB / 16 KB
     static constexpr uint32_t kStageBytes = kABytes + kBBytes;           // 48 KB / 32 KB
     static constexpr int kStages = kCg == 1 ? 4 : 6;
-    static constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kStages * kStageBytes + 512 /*barriers*/;
+    static constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kStages * kStageBytes + kControlBytes;
 };
 
 // ---- thin PTX wrappers -------------------------------------------------------------------------
@@ -361,6 +364,11 @@ struct SharedLayout {
     uint64_t mode;               // epilogue warps -> MMA issuer and epilogue: magnitude counts published
     uint64_t mag_counts[2 * kEpilogueWarps];   // per epilogue warp of the unit: see pack_magnitude_counts
     ScorePlan plan2;             // second pass: the plan derived from the number of marked rows
+    // 8-bit operands: the scales of a vocabulary tile's 256 columns, staged by the epilogue warps (32 columns
+    // each) when they start the tile.  Four buffers: the warps of a CTA are never more than three tiles apart
+    // (a warp starts tile t + 2 only after every warp has drained tile t - 1 from tensor memory).
+    uint64_t wscale_full[kScaleBufs];
+    alignas(16) float wscale[kScaleBufs][kBlockN];
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
@@ -491,6 +499,7 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
             mbar_init(smem_u32(&sh->acc_empty[b]), kEpilogueWarps * kCg);   // one arrival per epilogue warp
         }
         mbar_init(smem_u32(&sh->mode), kEpilogueWarps * kCg);
+        for (int b = 0; b < kScaleBufs; ++b) mbar_init(smem_u32(&sh->wscale_full[b]), kEpilogueWarps);
         sh->abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -709,6 +718,7 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
         const uint32_t acc_empty0 = (kCg == 2) ? mapa_shared(smem_u32(&sh->acc_empty[0]), 0u) : 0u;
         uint32_t chunk_count = 0;
         uint32_t mode_runs = 0;
+        uint32_t tile_count = 0;                             // vocabulary tiles so far (8-bit operands: scale buffers)
         bool ok = true;
         for (int w = 0; w < plan.waves && ok; ++w) {
             int st, nb, ne;
@@ -726,6 +736,9 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                                    ? token_ids[src] - plan.id_offset : -1;
             float row_scale = 0.0f;
             if (kFp8 && row < plan.rows) row_scale = (kSecond && compact) ? pass.scale_compact[row] : hidden_scale[src];
+            // what turns the values of `acc` below into base-2 exponents: log2(e), times the row's scale for 8-bit
+            // operands (whose column scales are applied first, the row's only here, in the same multiply-add)
+            const float to_exp2 = kFp8 ? row_scale * kLog2e : kLog2e;
             // state in base-2 units: run_max = max(z) * log2(e), run_sum = sum 2^(z*log2e - run_max)
             float run_max = -INFINITY, run_sum = 0.0f, picked = -INFINITY;
             for (int n = nb; n < ne && ok; ++n) {
@@ -738,6 +751,14 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                     ++mode_runs;
                     ck = adaptive_chunk_kblocks(read_magnitude_class<kCg>(sh), plan.chunk_kblocks, plan.k_blocks,
                                                 &assumed);
+                }
+                const uint32_t sbuf = tile_count % kScaleBufs;
+                if (kFp8) {
+                    // this warp's 32 of the tile's 256 column scales into shared memory (hidden behind the MMAs)
+                    const int c = (warp - 4) * 32 + lane, col = n * kBlockN + c;
+                    sh->wscale[sbuf][c] = col < plan.V ? __ldg(w_scale + col) : 0.0f;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sh->wscale_full[sbuf]));
                 }
                 float acc[kHalfN];                           // this thread's 128 logits of the tile
                 for (int kb0 = 0; kb0 < plan.k_blocks; kb0 += ck, ++chunk_count) {
@@ -780,13 +801,22 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                 if (!ok) break;
                 const int col_base = n * kBlockN + half * kHalfN;
                 if (kFp8) {
-                    // de-quantise: the sums are over codes; logit = sum * scale of the row * scale of the column
+                    // de-quantise: the sums are over codes; logit = sum * scale of the column * scale of the row.
+                    // The column scales come from shared memory, four at a time and the same for every lane; the
+                    // row's scale is folded into the exponent's multiply-add (to_exp2).
+                    if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&sh->wscale_full[sbuf]),
+                                                           (tile_count / kScaleBufs) & 1u, ab, kWaitLimitNs, true))) {
+                        ok = false;
+                        break;
+                    }
+                    const float4* ws4 = reinterpret_cast<const float4*>(&sh->wscale[sbuf][half * kHalfN]);
 #pragma unroll
-                    for (int j = 0; j < kHalfN; ++j) {
-                        const int col = col_base + j;
-                        acc[j] *= row_scale * (col < plan.V ? __ldg(w_scale + col) : 0.0f);
+                    for (int q = 0; q < kHalfN / 4; ++q) {
+                        const float4 sc = ws4[q];
+                        acc[4 * q] *= sc.x; acc[4 * q + 1] *= sc.y; acc[4 * q + 2] *= sc.z; acc[4 * q + 3] *= sc.w;
                     }
                 }
+                ++tile_count;
                 if (adapt_run && n == nb) {
                     // first tile of the run: publish how this warp's rows are spread over the magnitude classes
                     // to every CTA of the unit
@@ -794,6 +824,7 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
 #pragma unroll
                     for (int j = 0; j < kHalfN; ++j)
                         amax = (col_base + j < plan.V) ? fmaxf(amax, fabsf(acc[j])) : amax;
+                    if (kFp8) amax *= row_scale;
                     const uint64_t counts = pack_magnitude_counts(magnitude_class(amax));
                     if (lane == 0) {
                         const int slot = (int)rank * kEpilogueWarps + (warp - 4);
@@ -823,18 +854,19 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
                         if (rel < 32u) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) picked = (rel == (uint32_t)j) ? v[j] : picked;
+                            if (kFp8) picked *= row_scale;
                         }
                         float cmax = v[0];
 #pragma unroll
                         for (int j = 1; j < 32; ++j) cmax = fmaxf(cmax, v[j]);
-                        const float new_max = fmaxf(run_max, cmax * kLog2e);
+                        const float new_max = fmaxf(run_max, cmax * to_exp2);
                         run_sum *= ex2_approx(run_max - new_max);  // 2^-inf = 0 on the first group
                         run_max = new_max;
                         float acc0 = 0.0f, acc1 = 0.0f;
 #pragma unroll
                         for (int j = 0; j < 32; j += 2) {
-                            acc0 += ex2_approx(fmaf(v[j], kLog2e, -new_max));
-                            acc1 += ex2_approx(fmaf(v[j + 1], kLog2e, -new_max));
+                            acc0 += ex2_approx(fmaf(v[j], to_exp2, -new_max));
+                            acc1 += ex2_approx(fmaf(v[j + 1], to_exp2, -new_max));
                         }
                         run_sum += acc0 + acc1;
                     }
@@ -1045,7 +1077,7 @@ int launch_score_pass(specs_ctx* ctx, const ScorePlan& plan_in, bool second, con
                       const float* hidden_scale, const float* w_scale) {
     static_assert(Shape<1>::kSmemBytes <= 227 * 1024 && Shape<2>::kSmemBytes <= 227 * 1024, "shared memory budget");
     static_assert(Shape<1>::kStages <= kMaxStages && Shape<2>::kStages <= kMaxStages, "barrier arrays");
-    static_assert(sizeof(SharedLayout) <= 512, "barrier block");
+    static_assert(sizeof(SharedLayout) <= kControlBytes, "control block");
     const bool pair = plan_in.cta_group == 2;
     if (pair && (plan_in.units > ctx->pair_units || (plan_in.grid & 1))) return SPECS_ERR_CUDA;
     if (second && !plan_in.adaptive) return SPECS_OK;        // only adaptive plans mark rows

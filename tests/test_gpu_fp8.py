@@ -111,15 +111,6 @@ def test_fp8_scoring_at_the_7b_shape(ctx):
     qh, sh = F.quantize_rows(x.hidden[rows])
     want = F.token_logprobs_fp8(qh, sh, qw, sw, x.token_ids[rows])
     assert np.abs(got[rows] - want).max() <= TOK_ATOL
-    # timing, for the record of this test's log
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(50):
-        ctx.specs_score_blocks_fp8(hq, hs, wq, ws_, ids, off, tok, None, None, work)
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / 50
-    print(f"fp8 scoring of {x.rows} rows: {ms:.3f} ms per call, {2.0 * x.rows * cfg.d * cfg.vocab / ms / 1e9:.0f} TFLOP/s")
 
 
 def test_fused_fp8_step_equals_the_separate_calls_and_the_oracle(ctx):

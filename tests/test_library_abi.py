@@ -75,8 +75,8 @@ def test_plan_covers_every_tile_exactly_once(lib, rows, d, V, sms, cta_group):
     if p["rem_m"]:
         assert 1 <= p["split_rem"] and p["rem_m"] * p["split_rem"] <= p["units"]
     first = p["waves"] * p["grid"] * 2 * 3 * 128 * 4 + p["units"] * 8        # slots + progress words
-    if p["k_blocks"] <= p["chunk_kblocks"]:
-        assert p["workspace_bytes"] == first                      # one accumulation chunk: no second pass
+    if p["k_blocks"] <= p["chunk_kblocks"] or p["row_tiles"] <= 1:
+        assert p["workspace_bytes"] == first                      # one chunk, or one HBM-bound row tile: no second pass
         assert first < 256 * rows + (1 << 20)                     # never anything like rows x V
     else:
         # adaptive chunks: control block, list and gathered hidden states of the rows to re-score (at most
