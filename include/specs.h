@@ -560,7 +560,8 @@ int specs_score_plan_unit(int64_t rows, int32_t d, int32_t V, int32_t num_sms, i
  *
  *   status_word  device uint32 that receives SPECS_DEV_* bits by atomic OR (never
  *                cleared by the library); NULL sends them to an internal word that
- *                cannot be read back.
+ *                cannot be read back, so a NULL status word hides an expired wait
+ *                (SPECS_DEV_TIMEOUT) as well as a bad id: pass one if you can.
  *
  * Limits and sharing:
  *   - the plan for (rows, d, V) must fit the fixed scratch (waves x SMs x 3072 bytes
@@ -574,7 +575,13 @@ int specs_score_plan_unit(int64_t rows, int32_t d, int32_t V, int32_t num_sms, i
  *     e.g. on different streams, race on it: serialise them.
  *   - the first call on each device resolves the array's device address
  *     (cudaGetSymbolAddress) and the driver entry point it needs; make that first
- *     call before starting any stream capture. */
+ *     call before starting any stream capture.  With CUDA's default lazy module
+ *     loading that first call is also when the driver places the library's device
+ *     image, the array included, in device memory: a host whose own pool is about to
+ *     take the whole device must make the first call on each device BEFORE the pool
+ *     does (a call with rows = 0 and a non-NULL W_vocab is enough), or run with
+ *     CUDA_MODULE_LOADING=EAGER;
+ *     otherwise the first call fails with SPECS_ERR_CUDA. */
 #define SPECS_NOALLOC_SCRATCH_BYTES (8u << 20)
 int specs_score_blocks_noalloc(const void* hidden, const void* W_vocab, const int32_t* token_ids,
                                const int64_t* block_offsets, int64_t rows, int32_t d, int32_t V, int32_t B,
