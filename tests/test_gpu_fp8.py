@@ -76,6 +76,31 @@ def test_fp8_scoring_matches_its_definition(ctx, engine, blk, P, n, d, V):
     assert ctx.device_status() == 0
 
 
+def test_fp8_second_pass_rescoring_of_a_large_row(ctx):
+    # 8-bit operands with adaptive chunks (d beyond the 1024-element base chunk): one row 128 times larger than
+    # the rest is marked and re-scored from the compact buffer, with its gathered scale
+    d, V = 2048, 60000                                           # runs of six vocabulary tiles per work unit
+    cfg = I.StepConfig("f8fix", 7700, 1, 4, (80, 80), d, V, 1.0 / np.sqrt(d))
+    x = I.make_step_inputs(cfg)
+    big = x.hidden[123].copy()
+    nz = (big & 0x7f80) != 0
+    big[nz] += np.uint16(7 << 7)
+    x.hidden[123] = big
+    hq, hs = quantize_on_gpu(ctx, x.hidden)
+    wq, ws_ = quantize_on_gpu(ctx, x.w_vocab)
+    tok = torch.full((x.rows,), float("nan"), dtype=torch.float32, device=DEV)
+    work = torch.empty(ctx.score_workspace_bytes_fp8(x.rows, d, V), dtype=torch.uint8, device=DEV)
+    ctx.specs_score_blocks_fp8(hq, hs, wq, ws_, torch.from_numpy(x.token_ids).to(DEV),
+                               torch.from_numpy(x.block_offsets).to(DEV), tok, None, None, work)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == binding.DEV_ACCUM_RANGE
+    qh, sh = F.quantize_rows(x.hidden)
+    qw, sw = F.quantize_rows(x.w_vocab)
+    want = F.token_logprobs_fp8(qh, sh, qw, sw, x.token_ids)
+    assert abs(want[123]) > 50
+    assert np.abs(tok.cpu().numpy() - want).max() <= TOK_ATOL
+
+
 def test_fp8_argument_checks(ctx):
     h = torch.zeros((4, 24), dtype=torch.uint8, device=DEV)       # d % 16 != 0
     s = torch.ones(4, dtype=torch.float32, device=DEV)

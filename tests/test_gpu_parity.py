@@ -530,6 +530,27 @@ def test_adaptive_chunks_rescore_rows_beyond_the_sampled_magnitude(ctx, case):
         assert np.all(np.abs(fixed - got) <= 1e-4 * np.maximum(1.0, np.abs(want)))
 
 
+@pytest.mark.parametrize("engine", TC_ENGINES)
+def test_second_pass_under_both_tile_shapes(ctx, engine):
+    # the second pass has its own instantiation per tile shape: one large row, and every row large, under each
+    d, V = 2048, 30000
+    cfg = small_config("adapt_shapes", (96, 96), 1, 4, d, V, seed=5310, w_sigma=1.0 / math.sqrt(d))
+    x = I.make_step_inputs(cfg)
+    for rows_scaled in (np.array([200]), np.arange(x.rows)):
+        y = I.make_step_inputs(cfg)
+        y.hidden = _scale_rows_by_128(x.hidden, rows_scaled)
+        want = O.token_logprobs(y.hidden, y.w_vocab, y.token_ids)
+        ctx.set_engine(engine)
+        try:
+            got = _score_only(ctx, y)
+        finally:
+            ctx.set_engine(binding.ENGINE_TCGEN05)
+        # every row large: the first tile already shows it, the base chunks are kept and nothing is re-scored
+        expect_bits = binding.DEV_ACCUM_RANGE if len(rows_scaled) == 1 else 0
+        assert ctx.device_status() == expect_bits
+        assert np.abs(got - want).max() <= TOK_ATOL
+
+
 def test_one_large_row_does_not_shorten_its_tiles_chunks(ctx):
     # 1 % of the rows 20 times larger (the stress recipe): only those rows are re-scored; the others
     # keep the chunk length their own magnitude allows, and all meet the tolerance
