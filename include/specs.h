@@ -112,9 +112,13 @@ int specs_set_engine(specs_ctx* ctx, int engine);
  *     turns out to lie beyond that class -- anywhere in the vocabulary, or because the
  *     row is one of the few far larger than its tile -- is marked, and a second launch
  *     of the scoring kernel re-scores the marked rows with 512-element chunks (all rows
- *     when more than about an eighth of them are marked), so the per-token error stays
- *     within 2e-3 whatever the data; SPECS_DEV_ACCUM_RANGE then reports that this
- *     happened.  Measured at d = 5120 against the exact result: at most 1.9e-4 per token
+ *     when more than about an eighth of them are marked); rows with |logit| of 1024 and
+ *     more, where even 512-element chunks would leave a few 1e-3, are marked whatever
+ *     chunks the first pass used, and the second pass halves its chunks for every
+ *     doubling of the largest magnitude (down to 64 elements).  The per-token error
+ *     thus stays within 2e-3 wherever the large logits sit, up to magnitudes where the
+ *     fp32 spacing of the logits themselves approaches the tolerance (several
+ *     thousand); SPECS_DEV_ACCUM_RANGE reports that rows were re-scored.  Measured at d = 5120 against the exact result: at most 1.9e-4 per token
  *     for logit spreads up to 48, where a single chunk would be off by 2.3e-3. */
 #define SPECS_ACCUM_ADAPTIVE (-1)
 int specs_set_accum_chunk(specs_ctx* ctx, int32_t k_elements);

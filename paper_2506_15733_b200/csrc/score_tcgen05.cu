@@ -418,9 +418,9 @@ __device__ __forceinline__ int read_magnitude_class(const SharedLayout* sh) {
 // loss per accumulation averages half a spacing, and of the partial sum's magnitude, not the final one's;
 // measured, the bias is about a quarter of it (-5e-3 at |logit| = 700, d = 5120, one chunk: bound 2e-2).
 // The chunk is never shorter than `base`.  `*bound` receives the magnitude up to which that holds (2^cls),
-// infinity when the base chunk is kept: nothing shorter exists, so there is nothing to re-score with.
+// the base chunk's own bound when the base chunk is kept (the second pass has shorter chunks for rows beyond it).
 __device__ __forceinline__ int adaptive_chunk_kblocks(int cls, int base, int k_blocks, float* bound) {
-    *bound = INFINITY;
+    *bound = kBaseChunkBound;
     if (cls > 10) return base;
     const float n_acc = ldexpf(1.0e-3f, 24 - cls);           // spacing of [2^(cls-1), 2^cls) is 2^(cls-24)
     int kb = (int)fminf(n_acc * 0.25f, 1.0e6f);              // four accumulations per k-block
@@ -484,8 +484,10 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
         const uint32_t marked = *reinterpret_cast<const volatile uint32_t*>(&pass.ctl->count);
         if (marked == 0u) return;                            // every CTA of the grid takes the same decision
         compact = marked <= (uint32_t)pass.cap_rows;
-        if (threadIdx.x == 0)
-            sh->plan2 = compact ? make_compact_plan(plan_in, (int64_t)marked) : make_inplace_fix_plan(plan_in);
+        if (threadIdx.x == 0) {
+            const float mag = __uint_as_float(*reinterpret_cast<const volatile uint32_t*>(&pass.ctl->max_mag_bits));
+            sh->plan2 = compact ? make_compact_plan(plan_in, (int64_t)marked, mag) : make_inplace_fix_plan(plan_in, mag);
+        }
     }
     const ScorePlan& plan = kSecond ? sh->plan2 : plan_in;   // (plan2 is read after the barrier below)
 
@@ -527,7 +529,10 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
         asm volatile("griddepcontrol.wait;" ::: "memory");
         // (No early launch of the dependents here: set up while this kernel still runs, the small kernels behind
         // it made a step about 4 us slower than when they are launched at its end.)
-        if (pass.ctl != nullptr && blockIdx.x == 0 && threadIdx.x == 0) pass.ctl->count = 0u;
+        if (pass.ctl != nullptr && blockIdx.x == 0 && threadIdx.x == 0) {
+            pass.ctl->count = 0u;
+            pass.ctl->max_mag_bits = 0u;
+        }
     }
 
     // Registers move from the control warpgroup (which needs few) to the two epilogue warpgroups
@@ -725,7 +730,9 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
             if (!plan_unit(plan, w, unit, &st, &nb, &ne)) continue;
             const bool adapt_run = plan.adaptive && (ne - nb) >= 3;
             int ck = plan.chunk_kblocks;                     // k-blocks per chunk of the current tile
-            float assumed = INFINITY;                        // magnitude the lengthened chunks were sized for
+            // magnitude up to which the chunks in use keep the tolerance: the base chunk's own bound until (and
+            // unless) the run lengthens its chunks; no claim, and no marking, outside adaptive plans
+            float assumed = (!kSecond && plan.adaptive) ? kBaseChunkBound : INFINITY;
             const int64_t row = (int64_t)(st * kCg + (int)rank) * kBlockM + row_in_tile;
             // the row of the caller's arrays behind this one: itself, or the marked row gathered here
             int64_t src = row;

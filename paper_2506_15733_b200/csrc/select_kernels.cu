@@ -156,6 +156,10 @@ merge_splits_kernel(const ScorePlan plan, const float* __restrict__ workspace,
         if (partials) partials[row] = make_float4(f.max2, (float)f.sum2, f.logit, 0.0f);
         else          tok_logprob[row] = fold_logprob(f, token_ids[row], plan.V, status);
         if (f.marked && col.ctl != nullptr) {
+            // the magnitude that got the row marked is at most the larger of its maximum and its drafted logit
+            float mag = fabsf(f.max2) * (float)kLn2;
+            if (f.logit != -INFINITY) mag = fmaxf(mag, fabsf(f.logit));
+            if (mag == mag) atomicMax(&col.ctl->max_mag_bits, __float_as_uint(fminf(mag, 3.0e38f)));
             const uint32_t at = atomicAdd(&col.ctl->count, 1u);
             if (at < (uint32_t)col.cap_rows) {
                 col.list[at] = (int32_t)row;
@@ -187,7 +191,8 @@ __device__ __forceinline__ int second_pass_rows(const ScorePlan& plan, const Fix
     const uint32_t n = *reinterpret_cast<const volatile uint32_t*>(&fix.ctl->count);
     if (n == 0u) return 0;
     *compact = n <= (uint32_t)fix.cap_rows;
-    *plan2 = *compact ? make_compact_plan(plan, (int64_t)n) : make_inplace_fix_plan(plan);
+    // (the chunk length of the second pass does not enter the layout of its slots: any magnitude will do here)
+    *plan2 = *compact ? make_compact_plan(plan, (int64_t)n, 0.0f) : make_inplace_fix_plan(plan, 0.0f);
     return *compact ? (int)n : (int)plan.rows;
 }
 

@@ -96,8 +96,23 @@ __host__ __device__ inline size_t plan_slot_bytes(const ScorePlan& p) {
 // the compact buffer holds: the second launch re-scores every row in place instead.
 struct FixCtl {
     uint32_t count;        // rows marked by the merge (may exceed the compact capacity)
-    uint32_t pad[3];
+    uint32_t max_mag_bits; // largest |logit| that mattered in a marked row, as the bits of a non-negative float
+    uint32_t pad[2];
 };
+
+// Magnitude up to which the base chunk (32 accumulations) keeps the accumulated truncation under 2e-3: rows
+// beyond it are marked even where the base chunk was kept, and the second pass shortens its chunks for them.
+constexpr float kBaseChunkBound = 1024.0f;
+
+// k-blocks per accumulation chunk of the second pass, from the largest magnitude among the marked rows: as many
+// accumulations (four per k-block) as keep count x fp32 spacing at that magnitude under 2e-3, at most `base`,
+// at least one k-block.
+__host__ __device__ inline int second_pass_chunk_kblocks(float mag, int base) {
+    if (!(mag >= kBaseChunkBound)) return base;
+    int kb = base;
+    for (float bound = kBaseChunkBound; mag >= bound && kb > 1; bound *= 2.0f) kb >>= 1;
+    return kb < 1 ? 1 : kb;
+}
 
 // The workspace: triple slots [waves x grid], one 64-bit progress word per unit, and for adaptive
 // plans the control block, the list of marked rows, their gathered hidden states (and, for 8-bit
@@ -132,8 +147,9 @@ inline WsLayout plan_layout(const ScorePlan& p) {
 // Plan of the second pass over `n` gathered rows (n <= cap_rows, so one wave): same tile shape and
 // vocabulary as `base`, every super tile live at once, the units shared out over vocabulary chunks,
 // base chunks throughout.
-__host__ __device__ inline ScorePlan make_compact_plan(const ScorePlan& base, int64_t n) {
+__host__ __device__ inline ScorePlan make_compact_plan(const ScorePlan& base, int64_t n, float mag) {
     ScorePlan p = base;
+    p.chunk_kblocks = second_pass_chunk_kblocks(mag, base.chunk_kblocks);
     p.rows = n;
     p.row_tiles = (int32_t)((n + kBlockM - 1) / kBlockM);
     p.super_tiles = (p.row_tiles + p.cta_group - 1) / p.cta_group;
@@ -146,8 +162,9 @@ __host__ __device__ inline ScorePlan make_compact_plan(const ScorePlan& base, in
     return p;
 }
 // The second pass over all rows in place: the first pass's geometry with the base chunks.
-__host__ __device__ inline ScorePlan make_inplace_fix_plan(const ScorePlan& base) {
+__host__ __device__ inline ScorePlan make_inplace_fix_plan(const ScorePlan& base, float mag) {
     ScorePlan p = base;
+    p.chunk_kblocks = second_pass_chunk_kblocks(mag, base.chunk_kblocks);
     p.adaptive = 0;
     return p;
 }

@@ -461,12 +461,13 @@ def test_adaptive_chunks_keep_the_tolerance_across_logit_magnitudes(ctx, sigma_z
     assert np.abs(got[binding.ACCUM_ADAPTIVE] - got[512]).max() <= TOK_ATOL / 4
 
 
-def _scale_rows_by_128(bits, rows):
-    """Exact multiplication by 128 of the given rows of a bf16 bit array (exponent + 7), zeros left alone."""
+def _scale_rows_by_128(bits, rows, log2_factor=7):
+    """Exact multiplication by 128 (or 2^log2_factor) of the given rows of a bf16 bit array (exponent + 7),
+    zeros left alone."""
     out = bits.copy()
     sel = out[rows]
     nz = (sel & 0x7f80) != 0
-    sel[nz] += np.uint16(7 << 7)
+    sel[nz] += np.uint16(log2_factor << 7)
     out[rows] = sel
     return out
 
@@ -549,6 +550,21 @@ def test_second_pass_under_both_tile_shapes(ctx, engine):
         expect_bits = binding.DEV_ACCUM_RANGE if len(rows_scaled) == 1 else 0
         assert ctx.device_status() == expect_bits
         assert np.abs(got - want).max() <= TOK_ATOL
+
+
+@pytest.mark.parametrize("log2_factor", [9, 10])
+def test_rows_beyond_the_base_chunks_range_get_shorter_chunks(ctx, log2_factor):
+    # |logit| in the thousands: even 512-element chunks would leave a few 1e-3 of truncation there, so such rows
+    # are marked whatever chunks the first pass used, and the second pass shortens its chunks to their magnitude
+    d, V = 5120, 60000
+    cfg = small_config("adapt_huge", (64, 64), 1, 4, d, V, seed=5320, w_sigma=1.0 / math.sqrt(d))
+    x = I.make_step_inputs(cfg)
+    x.hidden = _scale_rows_by_128(x.hidden, np.array([11, 200]), log2_factor)
+    want = O.token_logprobs(x.hidden, x.w_vocab, x.token_ids)
+    assert np.abs(want[[11, 200]]).min() > 500
+    got = _score_only(ctx, x)
+    assert ctx.device_status() == binding.DEV_ACCUM_RANGE
+    assert np.abs(got - want).max() <= TOK_ATOL
 
 
 def test_one_large_row_does_not_shorten_its_tiles_chunks(ctx):
