@@ -51,7 +51,13 @@ def load_peaks():
     if os.path.exists(path):
         with open(path) as f:
             p = json.load(f)
-        return {k: float(p[k]) for k in FALLBACK_PEAKS if k in p} | {"source": "measured"}
+        out = {k: float(p[k]) for k in FALLBACK_PEAKS if k in p} | {"source": "measured"}
+        # the SM clock the sustained peak was measured at (boards of this machine settle at different clocks under
+        # the same power limit, so a sustained figure is also compared per MHz)
+        mhz = (p.get("clocks_under_load") or {}).get("sm_mhz_median")
+        if mhz:
+            out["sustained_sm_mhz"] = float(mhz)
+        return out
     return dict(FALLBACK_PEAKS) | {"source": "fallback"}
 
 
@@ -297,7 +303,11 @@ def roofline_fields(flops, kernel_ms, clocks, peaks, nominal, dtype_name):
     kind = regime_of(clocks)
     peak = peaks["bf16_tflops_sustained"] if kind == "sustained" else peaks["bf16_tflops"]
     frac = lambda p: achieved / p if achieved else None
-    return {"achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": frac(peak),
+    at_equal_clock = None
+    if achieved and kind == "sustained" and clocks.get("sm_mhz") and peaks.get("sustained_sm_mhz"):
+        # time x clock: this kernel's throughput per MHz against the sustained peak's per MHz
+        at_equal_clock = (achieved / clocks["sm_mhz"]) / (peaks["bf16_tflops_sustained"] / peaks["sustained_sm_mhz"])
+    return {"achieved": achieved, "frac_of_sustained_at_equal_clock": at_equal_clock, "peak": peak, "unit": "TFLOP/s", "frac": frac(peak),
             "peak_kind": f"{dtype_name} {kind}, of {peaks['source']}: chosen from the clocks sampled during the timed "
                          f"region (median {clocks.get('sm_mhz')} MHz of {clocks.get('sm_max_mhz')}, power cap active in "
                          f"{clocks.get('sw_power_cap_samples', 0)} of {clocks.get('samples', 0)} samples)",
@@ -333,6 +343,7 @@ def add_sustained(out, wl, ranks, sampler, beta, tau, peaks, nominal, dtype_name
         "steps": n, "seconds": leg["total_ms"] * 1e-3, "ms_per_step": leg["total_ms"] / n,
         "tokens_per_s": wl.rows * n / (leg["total_ms"] * 1e-3), "kernel_ms": leg["kernel_ms"],
         "achieved": r["achieved"], "peak": peaks["bf16_tflops_sustained"], "frac": r["frac_of_sustained"],
+        "frac_at_equal_clock": r["frac_of_sustained_at_equal_clock"],
         "frac_of_burst": r["frac_of_burst"], "frac_of_nominal": r["frac_of_nominal"],
         "sm_mhz": leg["clocks"].get("sm_mhz"), "reasons": leg["clocks"].get("reasons"),
         "regime_observed": regime_of(leg["clocks"]),
@@ -485,7 +496,7 @@ def main():
     nominal = NOMINAL_BF16_TFLOPS
     dtype_name = "bf16"
     if args.fp8:                                             # E4M3 runs at twice the bf16 rate
-        peaks = {k: (2.0 * v if k.startswith("bf16") else v) for k, v in peaks.items()}
+        peaks = {k: (2.0 * v if k.startswith("bf16") else v) for k, v in peaks.items()}   # (the clock is not doubled)
         peaks["source"] = "measured bf16 x 2 (nominal fp8 : bf16 ratio)" if peaks["source"] == "measured" else "fallback x 2"
         nominal, dtype_name = 2.0 * NOMINAL_BF16_TFLOPS, "fp8"
         args.no_e2e = True
