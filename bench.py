@@ -447,6 +447,9 @@ def main():
     ap.add_argument("--oracle-blocks", type=int, default=16, help="whole blocks per CPU-oracle sample")
     ap.add_argument("--tile-lead", type=int, default=None,
                     help="pacing of the CTA pairs that stream the same W chunk, in vocabulary tiles (0: off; default: the library's)")
+    ap.add_argument("--engine", default="auto", choices=["auto", "1cta", "2cta"],
+                    help="tile shape of the scoring kernel: the planner's choice, single CTAs (128-row tiles) or CTA "
+                         "pairs (256-row tiles)")
     ap.add_argument("--time-every", type=int, default=4,
                     help="record CUDA events around the scoring kernel on every K-th step of the timed region "
                          "(an event between two kernels of a step keeps the second from being set up early, "
@@ -520,6 +523,8 @@ def main():
     ctx = binding.Context(local_rank)
     if args.tile_lead is not None:
         ctx.set_tile_lead(args.tile_lead)
+    if args.engine != "auto":
+        ctx.set_engine(binding.ENGINE_TCGEN05_1CTA if args.engine == "1cta" else binding.ENGINE_TCGEN05_2CTA)
     beta, tau = cfg.betas[0], cfg.taus[0]
     wl = Workload(ctx, cfg, x, dev, fp8=args.fp8)
     head = measure(wl, ranks, sampler, args.steps, args.warmup, beta, tau, peaks, nominal, dtype_name, world,
@@ -581,7 +586,8 @@ def main():
 
     if rank == 0:
         roofline = {"bound": "tensor",
-                    "kernel": ("score_tiles_pair" if wl_plan_pair(binding, x, cfg, ctx) else "score_tiles") +
+                    "kernel": ("score_tiles_pair" if (args.engine == "2cta" or (args.engine == "auto" and
+                                                       wl_plan_pair(binding, x, cfg, ctx))) else "score_tiles") +
                               ("_fp8_kernel" if args.fp8 else "_kernel")} | head["roofline"]
         roofline["traffic"] = None if args.fp8 else DRAM_TRAFFIC_BYTES.get(cfg.name)
         roofline["kernel_calls_timed"] = head["kernel_calls_timed"]

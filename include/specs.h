@@ -124,11 +124,14 @@ int specs_set_engine(specs_ctx* ctx, int engine);
 int specs_set_accum_chunk(specs_ctx* ctx, int32_t k_elements);
 
 /* Pacing of the CTAs (pairs) that stream the same chunk of W_vocab: with tiles > 0 one
- * of them starts vocabulary tile t only once all of them have started tile
- * t - tiles, so that each W tile is fetched from HBM once and served from L2 to the
- * others (default 1; measured on 65536 rows at d = 3584: HBM reads 137 GB without,
- * 29 GB with, for an ideal of 24 GB).  0 switches the pacing off.  The wait is advisory and bounded (it gives up
- * after 40 us per tile and for good after four expiries). */
+ * of them passes pace point t only once all of them have passed point t - tiles, so
+ * that each W tile is fetched from HBM once and served from L2 to the others.  A pace
+ * point is the start of a vocabulary tile; where a wave's hidden states plus two tiles
+ * of W per vocabulary chunk would not fit in about 50 MB of L2 (d = 5120, or many
+ * chunks), the library places two to four evenly spaced points per tile.  Default 1
+ * (measured on 65536 rows at d = 3584: HBM reads 147 GB without, 24.5 GB with, for an
+ * ideal of 24.4 GB); 0 switches the pacing off.  The wait is advisory and bounded (it
+ * gives up after 40 us per point and for good after four expiries). */
 int specs_set_tile_lead(specs_ctx* ctx, int32_t tiles);
 
 /* Number of SMs the context schedules over (the persistent grid is one CTA per SM,

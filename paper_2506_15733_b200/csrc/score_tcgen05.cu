@@ -561,60 +561,68 @@ __device__ __forceinline__ void score_tiles_body(const CUtensorMap& map_hidden, 
             // the units of this wave that stream the same vocabulary chunk
             const int gm_w = w < plan.full_waves ? plan.group_m : plan.rem_m;
             const int group0 = (unit / gm_w) * gm_w;
+            // pace points: the start of a vocabulary tile and, where the plan asks for more than one per tile,
+            // evenly spaced k-blocks inside it
+            const int points = plan.pace_points > 1 ? plan.pace_points : 1;
+            const int seg = (plan.k_blocks + points - 1) / points;
             for (int n = nb; n < ne && ok; ++n) {
-                if (pace && gm_w > 1) {
-                    const int t = n - nb;
-                    if (lane == 0 && SPECS_IN_BOUNDS(unit, plan.units, status))
-                        st_progress(progress + unit, pace_key(plan.epoch, w, t));
-                    if (t >= plan.lead_tiles) {
-                        const unsigned long long need = pace_key(plan.epoch, w, t - plan.lead_tiles);
-                        const unsigned long long t0 = global_timer_ns();
-                        for (;;) {
-                            unsigned long long lo = ~0ull;
-                            for (int i = lane; i < gm_w; i += 32) {
-                                const unsigned long long v = ld_progress(progress + group0 + i);
-                                // a word of another launch counts as "not started"
-                                const unsigned long long cur = (v >> 48) == (plan.epoch & 0xffffu) ? v : 0ull;
-                                lo = cur < lo ? cur : lo;
-                            }
+                const int wrow0 = n * kBlockN + (int)rank * S::kBRows;
+                for (int kb0 = 0, sidx = 0; kb0 < plan.k_blocks && ok; kb0 += seg, ++sidx) {
+                    if (pace && gm_w > 1) {
+                        const int t = (n - nb) * points + sidx;
+                        if (lane == 0 && SPECS_IN_BOUNDS(unit, plan.units, status))
+                            st_progress(progress + unit, pace_key(plan.epoch, w, t));
+                        if (t >= plan.lead_tiles) {
+                            const unsigned long long need = pace_key(plan.epoch, w, t - plan.lead_tiles);
+                            const unsigned long long t0 = global_timer_ns();
+                            for (;;) {
+                                unsigned long long lo = ~0ull;
+                                for (int i = lane; i < gm_w; i += 32) {
+                                    const unsigned long long v = ld_progress(progress + group0 + i);
+                                    // a word of another launch counts as "not started"
+                                    const unsigned long long cur = (v >> 48) == (plan.epoch & 0xffffu) ? v : 0ull;
+                                    lo = cur < lo ? cur : lo;
+                                }
 #pragma unroll
-                            for (int o = 16; o > 0; o >>= 1) {
-                                const unsigned long long other = __shfl_xor_sync(0xffffffffu, lo, o);
-                                lo = other < lo ? other : lo;
+                                for (int o = 16; o > 0; o >>= 1) {
+                                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, lo, o);
+                                    lo = other < lo ? other : lo;
+                                }
+                                const bool expired =
+                                    __shfl_sync(0xffffffffu, global_timer_ns() - t0 > kPaceLimitNs, 0);
+                                if (lo >= need) { expiries = 0; break; }
+                                if (expired) {
+                                    if (++expiries >= kPaceMaxExpiries) pace = false;
+                                    break;
+                                }
                             }
-                            const bool expired = __shfl_sync(0xffffffffu, global_timer_ns() - t0 > kPaceLimitNs, 0);
-                            if (lo >= need) { expiries = 0; break; }
-                            if (expired) {
-                                if (++expiries >= kPaceMaxExpiries) pace = false;
+                        }
+                    }
+                    if (lane == 0) {
+                        const int kb1 = min(kb0 + seg, plan.k_blocks);
+                        for (int kb = kb0; kb < kb1; ++kb) {
+                            if (!mbar_wait(smem_u32(&sh->empty[stage]), phase ^ 1u, ab, kWaitLimitNs, true)) {
+                                ok = false;
                                 break;
                             }
+                            const uint32_t a_dst = tiles_addr + stage * kStageBytes;
+                            const uint32_t bar = full0 + stage * 8u;
+                            if (kCg == 1) {
+                                mbar_arrive_expect_tx(bar, kStageBytes);
+                                tma_load_2d(a_dst, map_rows, kb * kElemsK, row0, bar);
+                                tma_load_2d(a_dst + kABytes, &map_w, kb * kElemsK, wrow0, bar);
+                            } else {
+                                // the leader expects both CTAs' bytes; the peer's may be counted first
+                                if (rank == 0) mbar_arrive_expect_tx(smem_u32(&sh->full[stage]), 2u * kStageBytes);
+                                tma_load_2d_pair(a_dst, map_rows, kb * kElemsK, row0, bar);
+                                tma_load_2d_pair(a_dst + kABytes, &map_w, kb * kElemsK, wrow0, bar);
+                            }
+                            ++issued;
+                            if (++stage == kStages) { stage = 0; phase ^= 1u; }
                         }
                     }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
                 }
-                if (lane == 0) {
-                    const int wrow0 = n * kBlockN + (int)rank * S::kBRows;
-                    for (int kb = 0; kb < plan.k_blocks; ++kb) {
-                        if (!mbar_wait(smem_u32(&sh->empty[stage]), phase ^ 1u, ab, kWaitLimitNs, true)) {
-                            ok = false;
-                            break;
-                        }
-                        const uint32_t a_dst = tiles_addr + stage * kStageBytes;
-                        const uint32_t bar = full0 + stage * 8u;
-                        if (kCg == 1) {
-                            mbar_arrive_expect_tx(bar, kStageBytes);
-                            tma_load_2d(a_dst, map_rows, kb * kElemsK, row0, bar);
-                            tma_load_2d(a_dst + kABytes, &map_w, kb * kElemsK, wrow0, bar);
-                        } else {
-                            // the leader expects both CTAs' bytes; the peer's may be counted first
-                            if (rank == 0) mbar_arrive_expect_tx(smem_u32(&sh->full[stage]), 2u * kStageBytes);
-                            tma_load_2d_pair(a_dst, map_rows, kb * kElemsK, row0, bar);
-                            tma_load_2d_pair(a_dst + kABytes, &map_w, kb * kElemsK, wrow0, bar);
-                        }
-                        ++issued;
-                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
-                    }
-                }
-                ok = __shfl_sync(0xffffffffu, ok, 0);
             }
         }
         if (lane == 0) {
@@ -1092,6 +1100,19 @@ int launch_score_pass(specs_ctx* ctx, const ScorePlan& plan_in, bool second, con
     ScorePlan plan = plan_in;
     plan.epoch = (launch_counter.fetch_add(1) % 0xfffeu) + 1u;  // never 0
     plan.lead_tiles = ctx->lead_tiles;
+    {
+        // Pace points per vocabulary tile: what the units of a wave keep live in L2 is the wave's hidden-state tiles
+        // plus, per vocabulary chunk, the W bytes between the slowest and the fastest unit of the chunk (up to two
+        // pace intervals).  One point per tile unless that exceeds about 50 MB (d = 5120: 31 + 31 MB; measured
+        // 1.55 x the algorithmic HBM reads), then two or more.
+        const double tile_w = (double)kBlockN * plan.d * plan.elem_bytes;
+        const int gm = plan.full_waves > 0 ? plan.group_m : plan.rem_m;
+        const int sp = plan.full_waves > 0 ? plan.split_full : plan.split_rem;
+        const double hidden_live = (double)gm * kBlockM * plan.cta_group * plan.d * plan.elem_bytes;
+        int points = 1;
+        while (points < 4 && hidden_live + 2.0 * sp * tile_w / points > 50.0e6) ++points;
+        plan.pace_points = points;
+    }
     plan.id_offset = id_offset;
     query_pair_units(ctx->device, ctx->num_sms);             // shared-memory opt-in for this device
     const bool fp8 = plan.elem_bytes == 1;

@@ -69,6 +69,7 @@ struct ScorePlan {
     int32_t chunk_kblocks; // k-blocks per fresh tensor-core accumulator (chunks are summed in registers)
     int32_t lead_tiles;    // > 0: a unit starts vocabulary tile t of a wave only once every unit that streams the
                            //      same W chunk has started tile t - lead_tiles (advisory, bounded wait)
+    int32_t pace_points;   // pace points per vocabulary tile (1: the tile's start only); lead_tiles counts these
     int32_t id_offset;     // vocabulary index of W_vocab's first row (a shard of a larger vocabulary); 0 normally
     uint32_t epoch;        // distinguishes this launch's progress words from older contents of the workspace
     int32_t adaptive;      // 1: from the third vocabulary tile of a run on, lengthen the chunks as far as the
