@@ -40,7 +40,12 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (read + write) of one launch of the first-pass scoring kernel, by workload, from hardware
 # counters of an earlier capture of the same kernel; absent (null in the output) where none was taken
 # or the kernel has changed since.
-DRAM_TRAFFIC_BYTES = {}
+DRAM_TRAFFIC_BYTES = {
+    "step7b": 1.0981e9 + 4.2e6,
+    "batched": 12.16e9 + 9.1e6,
+    "dual_target": 24.485e9 + 16.3e6,
+    "stress": 42.67e9 + 19.5e6,
+}
 
 PER_CONFIG = ("batched", "dual_draft", "dual_target", "stress", "tiny")
 SEVEN_B_SHAPED = ("step7b", "batched", "dual_target")
