@@ -594,7 +594,9 @@ def main():
                     "kernel": ("score_tiles_pair" if (args.engine == "2cta" or (args.engine == "auto" and
                                                        wl_plan_pair(binding, x, cfg, ctx))) else "score_tiles") +
                               ("_fp8_kernel" if args.fp8 else "_kernel")} | head["roofline"]
-        roofline["traffic"] = None if args.fp8 else DRAM_TRAFFIC_BYTES.get(cfg.name)
+        # the table holds captures of the default launch configuration of the full workloads only
+        default_launch = not args.fp8 and args.problems is None and args.engine == "auto" and args.tile_lead is None
+        roofline["traffic"] = DRAM_TRAFFIC_BYTES.get(cfg.name) if default_launch else None
         roofline["kernel_calls_timed"] = head["kernel_calls_timed"]
         largest = per_config.get("dual_target")
         line = {"metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
