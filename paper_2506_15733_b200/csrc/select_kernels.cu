@@ -64,12 +64,16 @@ __device__ __forceinline__ RowFold fold_row(const ScorePlan& plan, const float* 
 #pragma unroll
         for (int u = 0; u < kMergeBatch; ++u) {
             const bool live = s0 + u * step < splits;
-            const float* p = base + (size_t)(live ? s0 + u * step : s0) * stride;
-            const float m0 = __ldcg(p), s_0 = __ldcg(p + kBlockM), t0 = __ldcg(p + 2 * kBlockM);
-            const float m1 = __ldcg(p + kHalf), s_1 = __ldcg(p + kHalf + kBlockM), t1 = __ldcg(p + kHalf + 2 * kBlockM);
-            f.marked = f.marked || (live && (s_0 < 0.0f || s_1 < 0.0f));
-            v[u][0] = live ? m0 : -INFINITY; v[u][1] = live ? fabsf(s_0) : 0.0f; v[u][2] = live ? t0 : -INFINITY;
-            v[u][3] = live ? m1 : -INFINITY; v[u][4] = live ? fabsf(s_1) : 0.0f; v[u][5] = live ? t1 : -INFINITY;
+            // (splits past the end are not loaded: the loads below are predicated, not redirected)
+            float m0 = -INFINITY, s_0 = 0.0f, t0 = -INFINITY, m1 = -INFINITY, s_1 = 0.0f, t1 = -INFINITY;
+            if (live) {
+                const float* p = base + (size_t)(s0 + u * step) * stride;
+                m0 = __ldcg(p); s_0 = __ldcg(p + kBlockM); t0 = __ldcg(p + 2 * kBlockM);
+                m1 = __ldcg(p + kHalf); s_1 = __ldcg(p + kHalf + kBlockM); t1 = __ldcg(p + kHalf + 2 * kBlockM);
+            }
+            f.marked = f.marked || s_0 < 0.0f || s_1 < 0.0f;
+            v[u][0] = m0; v[u][1] = fabsf(s_0); v[u][2] = t0;
+            v[u][3] = m1; v[u][4] = fabsf(s_1); v[u][5] = t1;
         }
 #pragma unroll
         for (int u = 0; u < kMergeBatch; ++u) {
