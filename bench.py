@@ -242,7 +242,9 @@ class Workload:
         two_pass = self.plan["k_blocks"] > self.plan["chunk_kblocks"] and self.plan["row_tiles"] > 1
         # score tiles; merge of the vocabulary splits; second pass (adaptive chunks only); finish (block sums,
         # SubSample + switch)
-        self.launches_per_step = 4 if two_pass else 3
+        # (tiny steps without a second pass merge inside the finish kernel: two launches)
+        fused_merge = not two_pass and rows * max(self.plan["split_full"], self.plan["split_rem"]) <= 2048
+        self.launches_per_step = 4 if two_pass else (2 if fused_merge else 3)
         if fp8:
             self.w_q = torch.empty((V, d), dtype=torch.uint8, device=dev)
             self.w_s = torch.empty(V, dtype=torch.float32, device=dev)
@@ -629,7 +631,9 @@ def launches_of(binding, x, cfg, ctx, fp8) -> int:
     """Kernels of this library launched per step: score tiles, merge, finish, plus the second scoring pass
     when the plan has adaptive accumulation chunks, plus the quantisation of the hidden states for E4M3."""
     p = binding.score_plan(x.rows, cfg.d, cfg.vocab, ctx.sm_count())
-    return 3 + (1 if p["k_blocks"] > p["chunk_kblocks"] and p["row_tiles"] > 1 else 0) + (1 if fp8 else 0)
+    two_pass = p["k_blocks"] > p["chunk_kblocks"] and p["row_tiles"] > 1
+    fused_merge = not two_pass and x.rows * max(p["split_full"], p["split_rem"]) <= 2048
+    return (4 if two_pass else (2 if fused_merge else 3)) + (1 if fp8 else 0)
 
 
 if __name__ == "__main__":

@@ -49,10 +49,12 @@ struct DeviceGuard {
 // launch does.
 int score_rows(specs_ctx* ctx, const ScorePlan& plan, const void* hidden, const void* w_vocab,
                const int32_t* token_ids, void* workspace, cudaStream_t stream, int32_t id_offset,
-               const float* hidden_scale, const float* w_scale, float* tok_logprob, float* partials, bool defer_fix) {
+               const float* hidden_scale, const float* w_scale, float* tok_logprob, float* partials, bool defer_fix,
+               bool finish_may_merge = false) {
     int st = launch_score_tcgen05(ctx, plan, hidden, w_vocab, token_ids, workspace, stream, id_offset, hidden_scale,
                                   w_scale);
     if (st != SPECS_OK) return st;
+    if (finish_may_merge && merge_in_finish(plan)) return SPECS_OK;   // the finish kernel merges; no second pass exists
     st = launch_merge(ctx, plan, workspace, token_ids, tok_logprob, partials, hidden, hidden_scale, stream);
     if (st != SPECS_OK || !plan.adaptive) return st;
     st = launch_score_second_pass(ctx, plan, hidden, w_vocab, token_ids, workspace, stream, id_offset, hidden_scale,
@@ -401,13 +403,15 @@ int specs_beam_step_fp8(specs_ctx* ctx, const void* hidden, const uint8_t* W_q, 
         float* h_scale = reinterpret_cast<float*>(base + off_scale);
         st = launch_quantize_rows(hidden, rows, d, base, h_scale, stream);
         if (st != SPECS_OK) return st;
-        st = score_rows(ctx, plan, base, W_q, token_ids, ws, stream, 0, h_scale, W_scale, tok_logprob, nullptr, true);
+        st = score_rows(ctx, plan, base, W_q, token_ids, ws, stream, 0, h_scale, W_scale, tok_logprob, nullptr, true,
+                        true);
         if (st != SPECS_OK) return st;
     }
     return launch_finish_step(ctx, plan, rows > 0 ? fix_view(plan, ws) : kNoFix, nullptr, kNoFix, token_ids,
                               block_offsets, cand_offsets, P,
                               const_cast<float*>(gen_tok_logprob), reward, uniforms, beta, tau, tok_logprob,
-                              blk_logprob_f64, gen_blk_logprob_f64, weights, chosen, accept, nullptr, nullptr, 0, stream);
+                              blk_logprob_f64, gen_blk_logprob_f64, weights, chosen, accept, nullptr, nullptr, 0,
+                              rows > 0 && merge_in_finish(plan) ? reinterpret_cast<const float*>(ws) : nullptr, stream);
 }
 
 int specs_block_sums(specs_ctx* ctx, const float* per_token, const int64_t* block_offsets, int32_t B, float* out,
@@ -520,14 +524,15 @@ int specs_beam_step(specs_ctx* ctx, const void* hidden, const void* W_vocab, con
     if (rows > 0) {
         if (workspace_bytes < plan_workspace_bytes(plan)) return SPECS_ERR_WORKSPACE;
         st = score_rows(ctx, plan, hidden, W_vocab, token_ids, workspace, stream, 0, nullptr, nullptr, tok_logprob,
-                        nullptr, true);
+                        nullptr, true, true);
         if (st != SPECS_OK) return st;
     }
     // the finish kernel only reads the generator's log-probabilities on this route
     return launch_finish_step(ctx, plan, rows > 0 ? fix_view(plan, workspace) : kNoFix, nullptr, kNoFix, token_ids,
                               block_offsets, cand_offsets, P, const_cast<float*>(gen_tok_logprob), reward, uniforms,
                               beta, tau, tok_logprob, blk_logprob_f64, gen_blk_logprob_f64, weights, chosen, accept,
-                              nullptr, nullptr, 0, stream);
+                              nullptr, nullptr, 0,
+                              rows > 0 && merge_in_finish(plan) ? static_cast<const float*>(workspace) : nullptr, stream);
 }
 
 size_t specs_beam_step_dual_workspace_bytes(const specs_ctx* ctx, int64_t rows, int32_t d_target, int32_t d_gen,
@@ -588,7 +593,7 @@ int specs_beam_step_dual(specs_ctx* ctx, const void* hidden_target, const void* 
                               rows > 0 ? fix_view(plan_g, ws_g) : kNoFix, token_ids, block_offsets,
                               cand_offsets, P, gen_tok_logprob, reward, uniforms, beta, tau, tok_logprob,
                               blk_logprob_f64, gen_blk_logprob_f64, weights, chosen, accept, chosen_ids, chosen_len,
-                              chosen_stride, stream);
+                              chosen_stride, nullptr, stream);
 }
 
 int specs_gather_chosen(specs_ctx* ctx, const int32_t* token_ids, const int64_t* block_offsets,

@@ -112,6 +112,26 @@ __device__ __forceinline__ float fold_logprob(const RowFold& f, int32_t id, int3
     return (float)((double)f.logit - lse);
 }
 
+constexpr int kMergeLanes = 4;                              // lanes that share a row's splits
+
+// A row's fold by kMergeLanes adjacent lanes of a warp: lane `sub` of the group takes every kMergeLanes-th split,
+// two shuffles combine them; every lane of the warp must call it, all lanes of a group receive the result.
+// A group with `active` false loads nothing (its result is empty) but still takes part in the shuffles.
+__device__ __forceinline__ RowFold fold_row_lanes(const ScorePlan& plan, const float* __restrict__ workspace,
+                                                  int64_t row, int sub, uint32_t* status, bool active = true) {
+    RowFold f = fold_row(plan, workspace, row, active ? sub : (1 << 30), kMergeLanes, status);
+#pragma unroll
+    for (int o = 1; o < kMergeLanes; o <<= 1) {
+        RowFold g;
+        g.max2 = __shfl_xor_sync(kFull, f.max2, o);
+        g.sum2 = __shfl_xor_sync(kFull, f.sum2, o);
+        g.logit = __shfl_xor_sync(kFull, f.logit, o);
+        g.marked = __shfl_xor_sync(kFull, (int)f.marked, o) != 0;
+        f = combine_folds(f, g);
+    }
+    return f;
+}
+
 // What the merge needs to collect the marked rows of an adaptive plan (ctl == NULL otherwise).
 struct CollectArgs {
     FixCtl* ctl;
@@ -124,7 +144,6 @@ struct CollectArgs {
     int32_t cap_rows;
 };
 constexpr int kMergeThreads = 128;
-constexpr int kMergeLanes = 4;                              // lanes that share a row's splits in merge_splits_kernel
 constexpr int kMergeRows = kMergeThreads / kMergeLanes;     // rows per CTA there
 
 // Four lanes per row, each folding every fourth split, then combined by shuffles: fold the first pass's splits and write the row's log-probability (or, for a holder
@@ -146,16 +165,7 @@ merge_splits_kernel(const ScorePlan plan, const float* __restrict__ workspace,
     // rows past the end fold row 0 (the shuffles below need every lane) and write nothing
     const int64_t row_raw = (int64_t)blockIdx.x * kMergeRows + threadIdx.x / kMergeLanes;
     const int64_t row = row_raw < plan.rows ? row_raw : 0;
-    RowFold f = fold_row(plan, workspace, row, sub, kMergeLanes, status);
-#pragma unroll
-    for (int o = 1; o < kMergeLanes; o <<= 1) {
-        RowFold g;
-        g.max2 = __shfl_xor_sync(kFull, f.max2, o);
-        g.sum2 = __shfl_xor_sync(kFull, f.sum2, o);
-        g.logit = __shfl_xor_sync(kFull, f.logit, o);
-        g.marked = __shfl_xor_sync(kFull, (int)f.marked, o) != 0;
-        f = combine_folds(f, g);
-    }
+    const RowFold f = fold_row_lanes(plan, workspace, row, sub, status, row_raw < plan.rows);
     if (row_raw < plan.rows && sub == 0) {
         if (partials) partials[row] = make_float4(f.max2, (float)f.sum2, f.logit, 0.0f);
         else          tok_logprob[row] = fold_logprob(f, token_ids[row], plan.V, status);
@@ -462,6 +472,8 @@ __device__ __forceinline__ void apply_second_pass(const ScorePlan& plan, const F
 
 // tok_logprob (and, with two scoring passes, gen_tok) hold the merged first-pass results; gen_tok may also
 // be the caller's own array of generator log-probabilities (fix_g.ctl == NULL then), or NULL.
+// With merge_slots the merge has not run: the CTA folds its problem's rows itself first (small steps without
+// a second pass, where a merge launch of its own would cost more than it does).
 __global__ void __launch_bounds__(kFinishThreads)
 finish_step_kernel(const ScorePlan plan, const FixView fix_t, const ScorePlan plan_g, const FixView fix_g,
                    const int32_t* __restrict__ token_ids, const int64_t* __restrict__ block_offsets,
@@ -469,7 +481,7 @@ finish_step_kernel(const ScorePlan plan, const FixView fix_t, const ScorePlan pl
                    const float* __restrict__ uniforms, float beta, float tau, float* tok_logprob, double* blk_lp,
                    double* gen_lp, float* __restrict__ weights, int32_t* chosen, uint8_t* __restrict__ accept,
                    int32_t* __restrict__ chosen_ids, int32_t* __restrict__ chosen_len, int32_t chosen_stride,
-                   uint32_t* __restrict__ status) {
+                   const float* __restrict__ merge_slots, uint32_t* __restrict__ status) {
     // Launched with programmatic stream serialisation: wait here for the kernels before it.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // let the next kernel of the stream (the next step's scoring kernel) begin its prologue
@@ -479,6 +491,16 @@ finish_step_kernel(const ScorePlan plan, const FixView fix_t, const ScorePlan pl
     const int a = cand_offsets[p], b = cand_offsets[p + 1];
     if (b > a) {
         const int64_t row_a = block_offsets[a], row_b = block_offsets[b];   // the problem's rows are contiguous
+        if (merge_slots != nullptr) {
+            const int sub = threadIdx.x % kMergeLanes;
+            for (int64_t r0 = row_a; r0 < row_b; r0 += kFinishThreads / kMergeLanes) {
+                const int64_t row_raw = r0 + threadIdx.x / kMergeLanes;
+                const int64_t row = row_raw < row_b ? row_raw : row_a;      // idle groups: a valid row, no loads
+                const RowFold f = fold_row_lanes(plan, merge_slots, row, sub, status, row_raw < row_b);
+                if (row_raw < row_b && sub == 0) tok_logprob[row] = fold_logprob(f, token_ids[row], plan.V, status);
+            }
+            __syncthreads();
+        }
         if (fix_t.ctl != nullptr || fix_g.ctl != nullptr) {
             apply_second_pass(plan, fix_t, row_a, row_b, token_ids, tok_logprob, status, threadIdx.x, kFinishThreads);
             apply_second_pass(plan_g, fix_g, row_a, row_b, token_ids, gen_tok, status, threadIdx.x, kFinishThreads);
@@ -622,12 +644,12 @@ int launch_finish_step(specs_ctx* ctx, const ScorePlan& plan, const FixView& fix
                        const int32_t* cand_offsets, int32_t P, float* gen_tok, const float* reward,
                        const float* uniforms, float beta, float tau, float* tok_logprob, double* blk_lp, double* gen_lp,
                        float* weights, int32_t* chosen, uint8_t* accept, int32_t* chosen_ids, int32_t* chosen_len,
-                       int32_t chosen_stride, cudaStream_t stream) {
+                       int32_t chosen_stride, const float* merge_slots, cudaStream_t stream) {
     if (P == 0) return SPECS_OK;
     const ScorePlan second = plan_g ? *plan_g : plan;
     return launch_chained(finish_step_kernel, (unsigned)P, kFinishThreads, stream, plan, fix_t, second, fix_g,
                           token_ids, block_offsets, cand_offsets, gen_tok, reward, uniforms, beta, tau, tok_logprob,
-                          blk_lp, gen_lp, weights, chosen, accept, chosen_ids, chosen_len, chosen_stride,
+                          blk_lp, gen_lp, weights, chosen, accept, chosen_ids, chosen_len, chosen_stride, merge_slots,
                           ctx->d_status);
 }
 

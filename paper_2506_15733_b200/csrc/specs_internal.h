@@ -278,12 +278,20 @@ int launch_fix_merge(specs_ctx* ctx, const ScorePlan& plan, const void* workspac
                      float* tok_logprob, float* partials, cudaStream_t stream);
 // Block sums of both per-token arrays, SubSample, the switch test and the gather of the chosen block, one CTA
 // per problem.  fix_t / fix_g: second-pass results still to be written over tok_logprob / gen_tok first.
+// merge_slots: the first pass's slots when no merge kernel ran (the CTAs then merge their own rows first).
 int launch_finish_step(specs_ctx* ctx, const ScorePlan& plan, const FixView& fix_t, const ScorePlan* plan_g,
                        const FixView& fix_g, const int32_t* token_ids, const int64_t* block_offsets,
                        const int32_t* cand_offsets, int32_t P, float* gen_tok, const float* reward,
                        const float* uniforms, float beta, float tau, float* tok_logprob, double* blk_lp, double* gen_lp,
                        float* weights, int32_t* chosen, uint8_t* accept, int32_t* chosen_ids, int32_t* chosen_len,
-                       int32_t chosen_stride, cudaStream_t stream);
+                       int32_t chosen_stride, const float* merge_slots, cudaStream_t stream);
+// Steps whose merge the finish kernel does itself (merge_slots): no second pass to wait for, and so few partial
+// triples (rows x vocabulary chunks) that one CTA per problem folds them faster than another launch would take
+// (64 rows x 4 chunks: 28 us per step instead of 32; 64 rows x 119 chunks: no gain, 128 x 119: 3 us slower).
+inline bool merge_in_finish(const ScorePlan& plan) {
+    const int splits = plan.split_full > plan.split_rem ? plan.split_full : plan.split_rem;
+    return !plan.adaptive && plan.rows * splits <= 2048;
+}
 int launch_gather_chosen(const int32_t* token_ids, const int64_t* block_offsets, const int32_t* cand_offsets,
                          const int32_t* chosen, int32_t P, int32_t* chosen_ids, int32_t* chosen_len, int32_t stride,
                          cudaStream_t stream);
