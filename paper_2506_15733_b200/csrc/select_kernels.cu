@@ -112,16 +112,25 @@ __device__ __forceinline__ float fold_logprob(const RowFold& f, int32_t id, int3
     return (float)((double)f.logit - lse);
 }
 
-constexpr int kMergeLanes = 4;                              // lanes that share a row's splits
+// Lanes that share a row's splits: four, or as many (a power of two, at most a warp) as leave a lane no more than
+// one batch of splits -- a plan for a few rows cuts the vocabulary into up to 148 chunks, and four lanes would fold
+// them in five dependent round trips to L2.  A function of the plan alone, so that every route that merges a plan
+// (merge kernel, finish kernel) combines the splits in the same order and gives the same bits.
+__host__ __device__ inline int merge_lanes(const ScorePlan& plan) {
+    const int splits = plan.split_full > plan.split_rem ? plan.split_full : plan.split_rem;
+    int lanes = 4;
+    while (lanes < 32 && splits > lanes * kMergeBatch) lanes <<= 1;
+    return lanes;
+}
 
-// A row's fold by kMergeLanes adjacent lanes of a warp: lane `sub` of the group takes every kMergeLanes-th split,
-// two shuffles combine them; every lane of the warp must call it, all lanes of a group receive the result.
+// A row's fold by `lanes` adjacent lanes of a warp: lane `sub` of the group takes every lanes-th split, shuffles
+// combine them; every lane of the warp must call it, all lanes of a group receive the result.
 // A group with `active` false loads nothing (its result is empty) but still takes part in the shuffles.
 __device__ __forceinline__ RowFold fold_row_lanes(const ScorePlan& plan, const float* __restrict__ workspace,
-                                                  int64_t row, int sub, uint32_t* status, bool active = true) {
-    RowFold f = fold_row(plan, workspace, row, active ? sub : (1 << 30), kMergeLanes, status);
-#pragma unroll
-    for (int o = 1; o < kMergeLanes; o <<= 1) {
+                                                  int64_t row, int sub, int lanes, uint32_t* status,
+                                                  bool active = true) {
+    RowFold f = fold_row(plan, workspace, row, active ? sub : (1 << 30), lanes, status);
+    for (int o = 1; o < lanes; o <<= 1) {
         RowFold g;
         g.max2 = __shfl_xor_sync(kFull, f.max2, o);
         g.sum2 = __shfl_xor_sync(kFull, f.sum2, o);
@@ -144,9 +153,9 @@ struct CollectArgs {
     int32_t cap_rows;
 };
 constexpr int kMergeThreads = 128;
-constexpr int kMergeRows = kMergeThreads / kMergeLanes;     // rows per CTA there
+constexpr int kMergeMaxRows = kMergeThreads / 4;            // rows per CTA with the fewest lanes per row
 
-// Four lanes per row, each folding every fourth split, then combined by shuffles: fold the first pass's splits and write the row's log-probability (or, for a holder
+// merge_lanes(plan) lanes per row, each folding its share of the splits, then combined by shuffles: fold the first pass's splits and write the row's log-probability (or, for a holder
 // of one vocabulary shard, its partials: max in base-2 units, sum of 2^(x - max), drafted id's logit or
 // -inf, 0).  A marked row also takes the next place in the list of rows to re-score; then the CTA's
 // threads together copy the hidden states of the CTA's marked rows into the compact buffer.  Rows beyond
@@ -155,17 +164,18 @@ __global__ void __launch_bounds__(kMergeThreads)
 merge_splits_kernel(const ScorePlan plan, const float* __restrict__ workspace,
                     const int32_t* __restrict__ token_ids, float* __restrict__ tok_logprob,
                     float4* __restrict__ partials, const CollectArgs col, uint32_t* __restrict__ status) {
-    __shared__ int32_t marked_row[kMergeRows], marked_at[kMergeRows];
+    __shared__ int32_t marked_row[kMergeMaxRows], marked_at[kMergeMaxRows];
     __shared__ int marked_n;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (threadIdx.x == 0) marked_n = 0;
     __syncthreads();
     asm volatile("griddepcontrol.wait;" ::: "memory");       // the scoring kernel's results
-    const int sub = threadIdx.x % kMergeLanes;
-    // rows past the end fold row 0 (the shuffles below need every lane) and write nothing
-    const int64_t row_raw = (int64_t)blockIdx.x * kMergeRows + threadIdx.x / kMergeLanes;
+    const int lanes = merge_lanes(plan);
+    const int sub = threadIdx.x % lanes;
+    // rows past the end load nothing and write nothing (the shuffles need every lane)
+    const int64_t row_raw = (int64_t)blockIdx.x * (kMergeThreads / lanes) + threadIdx.x / lanes;
     const int64_t row = row_raw < plan.rows ? row_raw : 0;
-    const RowFold f = fold_row_lanes(plan, workspace, row, sub, status, row_raw < plan.rows);
+    const RowFold f = fold_row_lanes(plan, workspace, row, sub, lanes, status, row_raw < plan.rows);
     if (row_raw < plan.rows && sub == 0) {
         if (partials) partials[row] = make_float4(f.max2, (float)f.sum2, f.logit, 0.0f);
         else          tok_logprob[row] = fold_logprob(f, token_ids[row], plan.V, status);
@@ -492,11 +502,12 @@ finish_step_kernel(const ScorePlan plan, const FixView fix_t, const ScorePlan pl
     if (b > a) {
         const int64_t row_a = block_offsets[a], row_b = block_offsets[b];   // the problem's rows are contiguous
         if (merge_slots != nullptr) {
-            const int sub = threadIdx.x % kMergeLanes;
-            for (int64_t r0 = row_a; r0 < row_b; r0 += kFinishThreads / kMergeLanes) {
-                const int64_t row_raw = r0 + threadIdx.x / kMergeLanes;
+            const int lanes = merge_lanes(plan);
+            const int sub = threadIdx.x % lanes;
+            for (int64_t r0 = row_a; r0 < row_b; r0 += kFinishThreads / lanes) {
+                const int64_t row_raw = r0 + threadIdx.x / lanes;
                 const int64_t row = row_raw < row_b ? row_raw : row_a;      // idle groups: a valid row, no loads
-                const RowFold f = fold_row_lanes(plan, merge_slots, row, sub, status, row_raw < row_b);
+                const RowFold f = fold_row_lanes(plan, merge_slots, row, sub, lanes, status, row_raw < row_b);
                 if (row_raw < row_b && sub == 0) tok_logprob[row] = fold_logprob(f, token_ids[row], plan.V, status);
             }
             __syncthreads();
@@ -625,7 +636,8 @@ int launch_merge(specs_ctx* ctx, const ScorePlan& plan, void* workspace, const i
         col.row_bytes = plan.d * plan.elem_bytes;
         col.cap_rows = lay.cap_rows;
     }
-    const unsigned blocks = (unsigned)((plan.rows + kMergeRows - 1) / kMergeRows);
+    const int rows_per_cta = kMergeThreads / merge_lanes(plan);
+    const unsigned blocks = (unsigned)((plan.rows + rows_per_cta - 1) / rows_per_cta);
     return launch_chained(merge_splits_kernel, blocks, kMergeThreads, stream, plan,
                           static_cast<const float*>(workspace), token_ids, tok_logprob,
                           reinterpret_cast<float4*>(partials), col, ctx->d_status);
