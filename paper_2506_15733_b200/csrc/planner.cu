@@ -35,9 +35,14 @@ double fill_plan(ScorePlan* p, int32_t cta_group, int32_t units) {
     };
     double best = -1.0;
     const int s_max = units < p->vocab_tiles ? units : p->vocab_tiles;
+    // super tiles whose hidden states fit the L2 budget together (at least one)
+    int gm_cap = (int)(kPlanL2Budget / tile_bytes);
+    if (gm_cap < 1) gm_cap = 1;
     for (int s = 1; s <= s_max; ++s) {
-        const int gm = units / s;
-        if (gm > 1 && gm * tile_bytes > kPlanL2Budget) continue;
+        // as many super tiles per wave as the units and the L2 budget allow; when the vocabulary has fewer tiles
+        // than there are units, s cannot grow to use them all and some units stay idle
+        int gm = units / s;
+        if (gm > gm_cap) gm = gm_cap;
         const int full = p->super_tiles / gm;
         const int rem = p->super_tiles - full * gm;
         int s_rem = 0;

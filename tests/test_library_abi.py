@@ -57,6 +57,8 @@ PLAN_CASES = [
     (65536, 1536, 151936, 148), (65536, 3584, 151936, 148), (131072, 5120, 152064, 148),
     (1, 8, 8, 148), (129, 72, 1000, 148), (20000, 64, 1000, 148), (10000, 1536, 2048, 148),
     (777, 128, 300, 7), (5000, 4096, 70000, 132), (128 * 148 + 1, 64, 257, 148),
+    (636, 5120, 421, 148),           # few vocabulary tiles and wide rows: the units cannot all be used
+    (40000, 8192, 300, 148), (129, 5120, 256, 148),
 ]
 
 
@@ -155,4 +157,24 @@ def test_checked_build_exports_the_same_symbols_and_says_what_it_is(lib):
         assert hasattr(dbg, name), name
     dbg.specs_debug_build.restype = ctypes.c_int
     assert dbg.specs_debug_build() == 1
+
+
+def test_planner_always_produces_a_covering_plan_on_random_shapes(lib):
+    # every (rows, d, V) gets at least one wave, never more units than exist, and waves that add up to all
+    # super tiles; wide rows with a vocabulary of a few tiles once came out with no wave at all
+    import numpy as np
+    rng = np.random.Generator(np.random.Philox(key=[8800, 1]))
+    for _ in range(400):
+        rows = int(rng.integers(1, 200000))
+        d = 8 * int(rng.integers(1, 1100))
+        V = int(rng.integers(1, 200000)) if rng.random() < 0.7 else int(rng.integers(1, 2000))
+        sms = int(rng.choice([1, 7, 132, 148]))
+        for cg in (0, 1, 2):
+            p = binding.score_plan(rows, d, V, sms, cg)
+            assert p["waves"] >= 1, (rows, d, V, sms, cg, p)
+            assert p["full_waves"] * p["group_m"] + p["rem_m"] == p["super_tiles"], (rows, d, V, sms, cg, p)
+            if p["full_waves"]:
+                assert 1 <= p["group_m"] * p["split_full"] <= p["units"] and p["split_full"] <= p["vocab_tiles"]
+            if p["rem_m"]:
+                assert 1 <= p["rem_m"] * p["split_rem"] <= p["units"] and 1 <= p["split_rem"] <= p["vocab_tiles"]
 
