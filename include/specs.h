@@ -118,7 +118,10 @@ int specs_set_engine(specs_ctx* ctx, int engine);
  *     doubling of the largest magnitude (down to 64 elements).  The per-token error
  *     thus stays within 2e-3 wherever the large logits sit, up to magnitudes where the
  *     fp32 spacing of the logits themselves approaches the tolerance (several
- *     thousand); SPECS_DEV_ACCUM_RANGE reports that rows were re-scored.  Measured at d = 5120 against the exact result: at most 1.9e-4 per token
+ *     thousand); SPECS_DEV_ACCUM_RANGE reports that rows were re-scored.  Inputs of at
+ *     most 128 rows (a single row tile, bound by streaming W rather than by the tensor
+ *     pipe) always use 512-element chunks and have no second pass: they keep the
+ *     tolerance for |logit| below 1024, like any fixed 512-element setting.  Measured at d = 5120 against the exact result: at most 1.9e-4 per token
  *     for logit spreads up to 48, where a single chunk would be off by 2.3e-3. */
 #define SPECS_ACCUM_ADAPTIVE (-1)
 int specs_set_accum_chunk(specs_ctx* ctx, int32_t k_elements);
