@@ -99,6 +99,15 @@ def test_fp8_second_pass_rescoring_of_a_large_row(ctx):
     want = F.token_logprobs_fp8(qh, sh, qw, sw, x.token_ids)
     assert abs(want[123]) > 50
     assert np.abs(tok.cpu().numpy() - want).max() <= TOK_ATOL
+    # the fused 8-bit step quantises the hidden states itself and takes the second pass's results in its finish kernel
+    from tests.gpu_util import DeviceStep
+    s = DeviceStep(ctx, x)
+    work2 = torch.empty(ctx.beam_step_fp8_workspace_bytes(x.rows, d, V), dtype=torch.uint8, device=DEV)
+    ctx.specs_beam_step_fp8(s.hidden, wq, ws_, s.token_ids, s.block_offsets, s.cand_offsets, s.draft, s.reward,
+                            s.uniforms, 1.0, 0.6, s.tok_lp, s.blk_lp64, s.gen_blk64, s.weights, s.chosen, s.accept, work2)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == binding.DEV_ACCUM_RANGE
+    assert np.array_equal(s.tok_lp.cpu().numpy(), tok.cpu().numpy())
 
 
 def test_fp8_argument_checks(ctx):

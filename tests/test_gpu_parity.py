@@ -567,6 +567,47 @@ def test_rows_beyond_the_base_chunks_range_get_shorter_chunks(ctx, log2_factor):
     assert np.abs(got - want).max() <= TOK_ATOL
 
 
+def test_second_pass_reaches_the_shard_partials_and_the_two_head_step(ctx):
+    # one large row, long reductions: marked and re-scored (a) in a vocabulary shard, whose partials must then
+    # be the second pass's, and (b) in both heads of the two-head step, whose finish kernel takes both fix-ups
+    from paper_2506_15733_b200 import vocab_parallel as VP
+    d, V = 2048, 30000
+    cfg = small_config("fix_routes", (96, 96), 2, 4, d, V, seed=5330, w_sigma=1.0 / math.sqrt(d))   # 768 rows
+    x = I.make_step_inputs(cfg)
+    x.hidden = _scale_rows_by_128(x.hidden, np.array([150]))
+    want = O.token_logprobs(x.hidden, x.w_vocab, x.token_ids)
+    dev = "cuda:0"
+    s = DeviceStep(ctx, x)
+    # (a) two shards
+    parts = []
+    for rank in range(2):
+        v0, v1 = VP.shard_bounds(V, 2, rank)
+        local = torch.full((x.rows, 4), float("nan"), dtype=torch.float32, device=dev)
+        ws = torch.empty(ctx.score_workspace_bytes(x.rows, d, v1 - v0), dtype=torch.uint8, device=dev)
+        ctx.specs_score_partials(s.hidden, s.w_vocab[v0:v1], s.token_ids, v0, local, ws)
+        parts.append(local)
+    out = torch.full((x.rows,), 7.0, dtype=torch.float32, device=dev)
+    ctx.specs_merge_partials(torch.stack(parts), s.token_ids, V, out)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == binding.DEV_ACCUM_RANGE
+    assert np.abs(out.cpu().numpy() - want).max() <= TOK_ATOL
+    # (b) both heads: the generator's head is the target's own here (same hidden states and weights)
+    gen_tok = torch.full((x.rows,), float("nan"), dtype=torch.float32, device=dev)
+    ws = torch.empty(ctx.beam_step_dual_workspace_bytes(x.rows, d, d, V), dtype=torch.uint8, device=dev)
+    ids_out = torch.full((2, 96), -9, dtype=torch.int32, device=dev)
+    len_out = torch.full((2,), -9, dtype=torch.int32, device=dev)
+    ctx.specs_beam_step_dual(s.hidden, s.w_vocab, s.hidden, s.w_vocab, s.token_ids, s.block_offsets, s.cand_offsets,
+                             s.reward, s.uniforms, 1.0, 0.6, s.tok_lp, gen_tok, s.blk_lp64, s.gen_blk64, s.weights,
+                             s.chosen, s.accept, ws, ids_out, len_out)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == binding.DEV_ACCUM_RANGE
+    t, g = s.tok_lp.cpu().numpy(), gen_tok.cpu().numpy()
+    assert np.abs(t - want).max() <= TOK_ATOL and np.array_equal(t, g)
+    assert np.allclose(s.blk_lp64.cpu().numpy(), O.block_sums(t, x.block_offsets), rtol=1e-12)
+    # identical heads: the ratio drops out, the weights are softmax(beta r) (text after Eq. 1)
+    assert np.abs(s.weights.cpu().numpy() - O.weights(O.scores(None, None, x.reward, 1.0), x.cand_offsets)).max() < 1e-6
+
+
 def test_one_large_row_does_not_shorten_its_tiles_chunks(ctx):
     # 1 % of the rows 20 times larger (the stress recipe): only those rows are re-scored; the others
     # keep the chunk length their own magnitude allows, and all meet the tolerance
