@@ -117,7 +117,8 @@ __device__ __forceinline__ float fold_logprob(const RowFold& f, int32_t id, int3
 // them in five dependent round trips to L2.  A function of the plan alone, so that every route that merges a plan
 // (merge kernel, finish kernel) combines the splits in the same order and gives the same bits.
 __host__ __device__ inline int merge_lanes(const ScorePlan& plan) {
-    const int splits = plan.split_full > plan.split_rem ? plan.split_full : plan.split_rem;
+    // the split count of most rows: that of the full waves when there are any, else the last wave's
+    const int splits = plan.full_waves > 0 ? plan.split_full : plan.split_rem;
     int lanes = 4;
     while (lanes < 32 && splits > lanes * kMergeBatch) lanes <<= 1;
     return lanes;
