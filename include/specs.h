@@ -384,9 +384,9 @@ int specs_score_blocks_fp8(specs_ctx* ctx, const uint8_t* hidden_q, const float*
                            float* tok_logprob, float* blk_logprob, double* blk_logprob_f64,
                            void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* The whole beam step with the 8-bit head, in three launches: quantise the step's
- * hidden states (bf16 [rows, d] in), score them against the pre-quantised weight,
- * and the finish kernel of specs_beam_step.  Arguments as in specs_beam_step, with
+/* The whole beam step with the 8-bit head: quantise the step's hidden states (bf16
+ * [rows, d] in), then the chain of specs_beam_step on the codes (scoring against the
+ * pre-quantised weight, merge, second pass, finish kernel).  Arguments as in specs_beam_step, with
  * W_q / W_scale from specs_quantize_rows_e4m3; the workspace also holds the codes and
  * scales of the hidden states (specs_beam_step_fp8_workspace_bytes). */
 size_t specs_beam_step_fp8_workspace_bytes(const specs_ctx* ctx, int64_t rows, int32_t d, int32_t V);

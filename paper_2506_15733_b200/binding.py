@@ -377,7 +377,7 @@ class Context:
     def specs_beam_step(self, hidden, w_vocab, token_ids, block_offsets, cand_offsets, gen_tok_logprob, reward,
                         uniforms, beta, tau, tok_logprob, blk_logprob_f64, gen_blk_logprob_f64, weights, chosen,
                         accept, workspace):
-        """The whole step on device tensors in two launches (scoring kernel + per-problem finish kernel)."""
+        """The whole step on device tensors as one chain of launches (scoring, merge, second pass, finish)."""
         rows, d = hidden.shape
         V = w_vocab.shape[0]
         B = block_offsets.shape[0] - 1

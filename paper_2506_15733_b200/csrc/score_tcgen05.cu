@@ -45,21 +45,32 @@
 // divides that bias by the number of chunks.  Each restart costs a read of the accumulator out
 // of TMEM, which holds up the tensor pipe for about 500 clocks, so chunks are only as short as
 // the logits demand: with plan.adaptive the first two vocabulary tiles of a run use the base
-// chunk; the epilogue warps publish the largest |logit| of the first tile, and from the third
-// tile on the MMA issuer and the epilogue both derive the chunk length from it
+// chunk; the epilogue warps publish how their rows' largest |logit| of the first tile spread over
+// magnitude classes, and from the third tile on the MMA issuer and the epilogue both derive the
+// chunk length from the class that all but 1/32 of the tile's samples stay within
 // (adaptive_chunk_kblocks).  The hand-over is a barrier ("mode") on which every epilogue warp of
-// the unit arrives after writing its maximum into every CTA of the unit.
+// the unit arrives after writing its counts into every CTA of the unit.
+//
+// Two passes: a row in which a logit that matters lies beyond the magnitude its chunks were sized
+// for (or beyond 1024, the base chunk's own range) leaves the first pass marked (a negative sum).
+// The merge collects the marked rows and gathers their hidden states; the same kernel body,
+// instantiated as the second pass (template parameter kSecond), re-scores them with short chunks:
+// it reads the count first and returns at once when it is zero, derives its plan from the count on
+// the device, and scores either the gathered rows or, when they outnumber the gather buffer,
+// every row in place.
 //
 // Pacing: the units (CTAs or pairs) that own the same vocabulary chunk in a wave read the same W
 // tiles.  Only while they stay within about a tile of each other does a tile come from HBM once and
 // from L2 for the others; left alone they drift apart within milliseconds and every tile is fetched
 // several times.  Each unit therefore publishes its progress in a 64-bit word behind the workspace's
-// slots and does not start tile t before all units of its chunk have started tile t - lead.  The
-// wait is advisory (bounded, gives up for good after a few expiries).
+// slots and does not pass pace point t before all units of its chunk have passed point t - lead;
+// a pace point is the start of a vocabulary tile, or one of several evenly spaced k-blocks of a tile
+// where the wave's working set would otherwise outgrow L2 (plan.pace_points).  The wait is advisory
+// (bounded, gives up for good after a few expiries).
 //
 // 8-bit operands (template parameter kFp8): the same kernel on E4M3 codes with per-row scales,
-// 128 elements per k-block, tcgen05.mma kind::f8f6f4; the epilogue first multiplies each
-// accumulator by scale of the row x scale of the column.
+// 128 elements per k-block, tcgen05.mma kind::f8f6f4; the epilogue applies the column scales (staged
+// in shared memory per tile) to the accumulators and folds the row's scale into the exponent.
 //
 // Every mbarrier wait is bounded; on expiry the CTA raises SPECS_DEV_TIMEOUT, all roles leave
 // their loops, the producer waits (bounded) for its copies in flight, TMEM is freed and the
