@@ -156,11 +156,12 @@ struct CollectArgs {
 constexpr int kMergeThreads = 128;
 constexpr int kMergeMaxRows = kMergeThreads / 4;            // rows per CTA with the fewest lanes per row
 
-// merge_lanes(plan) lanes per row, each folding its share of the splits, then combined by shuffles: fold the first pass's splits and write the row's log-probability (or, for a holder
-// of one vocabulary shard, its partials: max in base-2 units, sum of 2^(x - max), drafted id's logit or
-// -inf, 0).  A marked row also takes the next place in the list of rows to re-score; then the CTA's
-// threads together copy the hidden states of the CTA's marked rows into the compact buffer.  Rows beyond
-// the buffer's capacity are only counted: the second pass then works on all rows in place.
+// merge_lanes(plan) lanes per row, each folding its share of the row's splits, combined by shuffles; lane 0 of
+// the group writes the row's log-probability (or, for a holder of one vocabulary shard, its partials: max in
+// base-2 units, sum of 2^(x - max), drafted id's logit or -inf, 0).  A marked row also takes the next place in
+// the list of rows to re-score; then the CTA's threads together copy the hidden states of the CTA's marked rows
+// into the compact buffer.  Rows beyond the buffer's capacity are only counted: the second pass then works on
+// all rows in place.
 __global__ void __launch_bounds__(kMergeThreads)
 merge_splits_kernel(const ScorePlan plan, const float* __restrict__ workspace,
                     const int32_t* __restrict__ token_ids, float* __restrict__ tok_logprob,
